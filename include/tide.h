@@ -1,0 +1,162 @@
+/* tide.h — C ABI of the tide-kv library (B200 / sm_100a only).
+ *
+ * The GPU hot path behind Continuous Task Batching (CTB, paper Section 4):
+ * rollout tasks that pause for an external environment keep their KV state
+ * resident and resume with the observation tokens appended, instead of
+ * re-running prefill over their history (paper Section 1, first challenge;
+ * Section 2.2).  Per engine step the GPU work is (a) appending each task's
+ * new K/V rows into a paged cache and (b) grouped-query attention of a mixed
+ * batch — one-token decode rows next to multi-token resume rows whose causal
+ * queries see the whole preserved prefix.
+ *
+ * Conventions
+ *   - One tide_kv_t per GPU (a rollout data-parallel rank is its own token
+ *     budget pool with its own cache, Section 4.1).  One caller thread per
+ *     tide_kv_t.  The CUDA device current at tide_kv_create must be current
+ *     at every later call.
+ *   - "host" pointers are ordinary host memory read during the call; "device"
+ *     pointers are device memory on that GPU, 16-byte aligned, owned by the
+ *     caller and never freed or reallocated by the library.
+ *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*);
+ *     host bookkeeping is updated before the call returns.  append followed by
+ *     attend on one stream is ordered.
+ *   - Every call returns TIDE_OK (0) or a negative tide_status_t.  All
+ *     validation happens before any mutation: a failing call changes nothing.
+ *     There is no CPU fallback anywhere.
+ *   - Values are bf16 (raw 16-bit patterns); accumulation is fp32.
+ */
+#ifndef TIDE_H_
+#define TIDE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TIDE_OK = 0,
+  TIDE_ERR_INVALID_ARG = -1,    /* NULL / misaligned pointer, bad geometry, bad indptr, bad layer      */
+  TIDE_ERR_UNKNOWN_TASK = -2,   /* task id not registered by tide_kv_alloc                             */
+  TIDE_ERR_TASK_EXISTS = -3,    /* tide_kv_alloc of a live task                                        */
+  TIDE_ERR_DUPLICATE_TASK = -4, /* the same task twice in one tide_kv_append                           */
+  TIDE_ERR_NO_PAGES = -5,       /* free pages cannot hold the request (the caller pauses or evicts,    */
+                                /* Algorithm 1, eviction loop)                                         */
+  TIDE_ERR_TABLE_FULL = -6,     /* a task would exceed max_pages_per_task                              */
+  TIDE_ERR_CTX_RANGE = -7,      /* a row violates 1 <= q_len <= ctx_len <= resident length             */
+  TIDE_ERR_WORKSPACE = -8,      /* pool / workspace / batch limits too small for the request           */
+  TIDE_ERR_CUDA = -9,           /* a CUDA runtime call failed                                          */
+  TIDE_ERR_DEVICE_TIMEOUT = -10 /* a bounded wait inside a kernel ran out (reported by tide_status)    */
+} tide_status_t;
+
+typedef struct tide_kv tide_kv_t; /* opaque */
+
+/* One batch row of tide_attend.  ctx_len is the number of cached tokens the row
+ * attends over INCLUDING this step's q_len appended tokens; the preserved
+ * prefix is ctx_len - q_len.  A decode row has q_len 1. */
+typedef struct {
+  int32_t task;
+  int32_t q_len;
+  int32_t ctx_len;
+} tide_row_t;
+
+typedef struct {
+  int32_t num_layers;         /* must be 1                                                          */
+  int32_t num_q_heads;        /* Hq, a multiple of num_kv_heads, Hq/Hkv <= 16                       */
+  int32_t num_kv_heads;       /* Hkv                                                                */
+  int32_t head_dim;           /* D: 64 or 128                                                       */
+  int32_t page_size;          /* S: 16 or 32 tokens                                                 */
+  int32_t max_tasks;          /* task ids are dense ints in [0, max_tasks)                          */
+  int32_t max_pages_per_task; /* page-table row length                                              */
+  int32_t max_batch_rows;     /* most rows / tasks in one tide_attend / tide_kv_append              */
+  int64_t num_pages;          /* pool capacity in pages                                             */
+  int64_t max_batch_tokens;   /* most query tokens in one tide_attend (sum of q_len) and most new   */
+                              /* tokens in one host-buffer step                                     */
+  void* pool;                 /* device; >= pool_bytes from tide_kv_required_bytes, 1024-B aligned  */
+  size_t pool_bytes;
+  void* workspace;            /* device scratch; >= workspace_bytes, 256-B aligned                  */
+  size_t workspace_bytes;
+  const int32_t* free_order;  /* host; permutation of [0, num_pages): the order in which a fresh    */
+                              /* pool hands pages out.  NULL = identity.                            */
+} tide_kv_config_t;
+
+/* Sizes the caller must provide for cfg's geometry (pool / workspace fields of cfg are ignored). */
+int tide_kv_required_bytes(const tide_kv_config_t* cfg, size_t* pool_bytes, size_t* workspace_bytes);
+
+/* Creates the cache object: host bookkeeping, a pinned staging ring, device tables carved from
+ * cfg->workspace.  The pool is NOT cleared.  Physical page layout inside the pool is private to the
+ * library; read logical content back with tide_kv_read. */
+int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out);
+int tide_kv_destroy(tide_kv_t* kv);
+
+/* Flush every task and restart the free stack from free_order (NULL = identity): the cache flush
+ * that follows each weight synchronisation (Section 5.2, rollout shrink / KV-cache reset). */
+int tide_kv_reset(tide_kv_t* kv, const int32_t* free_order);
+
+/* Register `task` with length 0 (Section 4.1, token-aware admission).  Takes no pages; pages are
+ * taken by tide_kv_append.  reserve_tokens is an admission check only: the call fails with
+ * TIDE_ERR_NO_PAGES unless free_pages * page_size >= reserve_tokens (0 = no check). */
+int tide_kv_alloc(tide_kv_t* kv, int32_t task, int64_t reserve_tokens);
+
+/* Append indptr[j+1]-indptr[j] tokens to task_ids[j] for j in [0, n_tasks) (the resume step of
+ * Section 4: observation tokens are added to the preserved state).  new_k / new_v: device bf16
+ * [T, Hkv, D], T = indptr[n_tasks], token rows of task j at [indptr[j], indptr[j+1]).
+ * Pages are popped from the free stack in array order, one each time a token lands on slot 0 of a
+ * new logical page.  All-or-nothing: on any error no task changes.  Zero-length entries are no-ops. */
+int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids /*host*/,
+                   const int32_t* indptr /*host, n_tasks+1*/, const void* new_k /*device*/,
+                   const void* new_v /*device*/, void* stream);
+
+/* Attention of a mixed continuous batch over the cache (Section 3.2: concurrent multi-task
+ * generation on one rank; Section 4: resumed tasks continue from preserved state).
+ * Row b: query i in [0, q_len) sits at position ctx_len - q_len + i and sees keys [0, that position]
+ * (causal inside the appended chunk, full attention to the preserved prefix).  Query head h reads KV
+ * head h / (Hq/Hkv).  q, out: device bf16 [sum q_len, Hq, D], rows concatenated in batch order;
+ * lse: device fp32 [sum q_len, Hq] (natural log of the sum of exp of scaled logits) or NULL.
+ * page_table: device int32 [max_tasks][max_pages_per_task] to read instead of the library's own
+ * table, or NULL.  The same task may appear in several rows.  Read-only on the cache. */
+int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows /*host*/,
+                const int32_t* page_table /*device or NULL*/, const void* q /*device*/, float scale,
+                void* out /*device*/, float* lse /*device or NULL*/, void* stream);
+
+/* One whole CTB step from HOST buffers: copies new_k / new_v / q to the device, appends q_len
+ * tokens to every row's task (rows must name distinct tasks; ctx_len must equal the resident length
+ * after the append), attends, and copies out / lse back.  new_k, new_v: host bf16 [sum q_len, Hkv, D];
+ * q, out: host bf16 [sum q_len, Hq, D]; lse: host fp32 or NULL.  Host buffers should be pinned for
+ * the copies to be asynchronous.  The call returns after the results have arrived. */
+int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows /*host*/,
+                   const void* new_k /*host*/, const void* new_v /*host*/, const void* q /*host*/,
+                   float scale, void* out /*host*/, float* lse /*host or NULL*/, void* stream);
+
+/* Return the task's pages to the free stack, last page first, and forget the task (task end or
+ * eviction, Algorithm 1).  Host only; page contents are not cleared. */
+int tide_kv_release(tide_kv_t* kv, int32_t task);
+
+/* Roll a live task back to new_len <= its length, returning pages ceil(new_len/S).. last-to-first
+ * (sliding-window pruning of old observations, Appendix C.2).  Host only. */
+int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len);
+
+/* Introspection (the per-rank token usage CTB schedules on, Section 4.1 / Algorithm 1). */
+int tide_kv_task_len(tide_kv_t* kv, int32_t task, int32_t* len);
+int tide_kv_page_table(tide_kv_t* kv, int32_t task, int32_t* out /*host*/, int32_t cap, int32_t* n_pages);
+int tide_kv_usage(tide_kv_t* kv, int64_t* used_tokens, int64_t* free_pages);
+/* Logical content of a task as contiguous device bf16 [len, Hkv, D] (out_k / out_v). */
+int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k /*device*/, void* out_v /*device*/,
+                 void* stream);
+
+/* Synchronises `stream` and returns the device status word: TIDE_OK, or TIDE_ERR_DEVICE_TIMEOUT if a
+ * bounded wait in a kernel ran out since the last call (the word is then cleared). */
+int tide_status(tide_kv_t* kv, void* stream);
+
+/* Counters of the most recent tide_attend: work items launched on the decode-style and the
+ * tensor-tile paths, rows merged, and kernels launched by the most recent append + attend pair. */
+int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,
+                   int64_t* kernel_launches);
+
+const char* tide_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TIDE_H_ */

@@ -1,0 +1,453 @@
+// Split-KV attention over the paged cache with warp-level tensor-core tiles (mma.sync) — the decode path,
+// and the general path for resume rows that the tcgen05 kernel does not take.
+//
+// What it computes (paper Section 4: a resumed task continues from its preserved KV state; the maths is
+// ordinary scaled-dot-product softmax attention with grouped KV heads): for a work item
+// (row, kv_head, m_tile, split) the online-softmax partial over keys [kv_begin, kv_end) for a tile of
+// packed rows r = q_index * G + g (the G query heads that share this KV head), query q_index seeing keys
+// [0, prefix + q_index].  K/V pages are read ONCE per KV head for all G query heads.
+//
+// Structure: one producer warp streams whole (page, head) blocks (K and V, contiguous in the pool) into a
+// ring of shared-memory stages with 1-D bulk copies that complete on mbarriers; four consumer warps run
+// m16n8k16 bf16 MMAs straight from the pre-swizzled blocks with ldmatrix.  Decode items: the four warps
+// split the keys of a stage and merge their (m, l, O) at the end.  Tile items: each warp owns 16 of the
+// 64 packed rows.  Bound by HBM bandwidth for decode: Hkv*D*4 bytes per context token, 4*D*Hq flops.
+#include <cfloat>
+#include <climits>
+
+#include "tide_internal.h"
+
+namespace tide {
+
+constexpr int kConsumerWarps = 4;
+constexpr int kAttendThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStages = 3;
+
+template <int D>
+struct MmaCfg {
+  static constexpr int kStageBytes = kStageKeys * D * 4;  // K + V, bf16
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+};
+
+__device__ __forceinline__ int blk_chunk_offset(int S, int slot, int c) {
+  return (c >> 3) * (S * 128) + slot * 128 + (((c & 7) ^ (slot & 7)) << 4);
+}
+
+template <int D, bool DECODE>
+__global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const AttendParams P) {
+  constexpr int KS = D / 16;                 // k-steps of Q.K^T
+  constexpr int NT = D / 8;                  // n-tiles of O
+  constexpr int STEP_KB = DECODE ? 1 : 4;    // 16-key blocks per softmax step of one warp
+  constexpr int TILE_M = DECODE ? kDecodeTileRows : kMmaTileRows;
+  constexpr int STAGE_BYTES = MmaCfg<D>::kStageBytes;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t s_full[kStages];
+  __shared__ __align__(8) uint64_t s_empty[kStages];
+  __shared__ int s_abort;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Geom& g = P.g;
+
+  // ---- which item ----
+  const int item = blockIdx.x;
+  const int si = find_segment(P.n_segs, item, [&](int i) { return P.segs[i].item_base; });
+  const Segment seg = P.segs[si];
+  int local = item - seg.item_base;
+  const int m_tile = local % seg.n_mtiles;
+  local /= seg.n_mtiles;
+  const int split = local % seg.n_splits;
+  const int kvh = local / seg.n_splits;
+  const int R = seg.n * g.G;                       // packed rows of this (row, kv head)
+  const int tile_row0 = m_tile * TILE_M;
+  const int r_last = min(R, tile_row0 + TILE_M) - 1;
+  const int kv_begin = split * seg.chunk;
+  const int kv_end = min(kv_begin + seg.chunk, seg.p + r_last / g.G + 1);
+  const bool direct = seg.n_splits == 1;
+  const float kLn2 = 0.6931471805599453f;
+
+  // rows this thread owns inside its warp's 16-row MMA tile
+  const int row_base = tile_row0 + (DECODE ? 0 : warp * 16);
+  const int r_lo = row_base + (lane >> 2), r_hi = r_lo + 8;
+  const bool v_lo = r_lo < R, v_hi = r_hi < R;
+  const int qi_lo = r_lo / g.G, qi_hi = r_hi / g.G;
+  const int hd_lo = kvh * g.G + (r_lo - qi_lo * g.G), hd_hi = kvh * g.G + (r_hi - qi_hi * g.G);
+
+  if (kv_end <= kv_begin) {
+    // nothing visible in this split (only possible when n_splits > 1): neutral partials
+    if (warp < kConsumerWarps && (lane & 3) == 0 && (!DECODE || warp == 0)) {
+      if (v_lo) P.part_lse[seg.part_base + (split * seg.n + qi_lo) * g.Hq + hd_lo] = -INFINITY;
+      if (v_hi) P.part_lse[seg.part_base + (split * seg.n + qi_hi) * g.Hq + hd_hi] = -INFINITY;
+    }
+    return;
+  }
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&s_empty[i]), kConsumerWarps);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  volatile int* abort_flag = &s_abort;
+
+  const int n_st = (kv_end - kv_begin + kStageKeys - 1) / kStageKeys;
+
+  if (warp == kConsumerWarps) {
+    // ================= producer warp =================
+    const int pages_per_stage = kStageKeys / g.S;
+    for (int st = 0; st < n_st; ++st) {
+      const int slot = st % kStages;
+      if (st >= kStages) mbar_wait(smem_u32(&s_empty[slot]), ((st / kStages) - 1) & 1, abort_flag, P.status);
+      const int key0 = kv_begin + st * kStageKeys;
+      const int npages = min(pages_per_stage, (kv_end - key0 + g.S - 1) / g.S);
+      const uint32_t bar = smem_u32(&s_full[slot]);
+      if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * g.head_bytes));
+      __syncwarp();
+      if (lane < npages) {
+        const long long page = P.table[seg.table_off + key0 / g.S + lane];
+        const uint8_t* src = P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes;
+        bulk_g2s(smem_base + slot * STAGE_BYTES + lane * g.head_bytes, src, (uint32_t)g.head_bytes, bar);
+      }
+    }
+    if (*abort_flag && lane == 0) {
+      // a wait gave up somewhere: do not leave the CTA while copies into its shared memory are in flight
+      for (int st = max(0, n_st - kStages); st < n_st; ++st) {
+        const uint32_t bar = smem_u32(&s_full[st % kStages]);
+        const long long t0 = global_ns();
+        while (!mbar_try(bar, (st / kStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    return;
+  }
+
+  // ================= consumer warps =================
+  const int kv_limit_lo = v_lo ? min(kv_end, seg.p + qi_lo + 1) : kv_end;  // keys j < limit are visible
+  const int kv_limit_hi = v_hi ? min(kv_end, seg.p + qi_hi + 1) : kv_end;
+  // last key any row of this warp can see, and the smallest limit (masking needed beyond it)
+  int w_end, w_min_limit;
+  {
+    const int wr_first = row_base, wr_last = min(R, row_base + 16) - 1;
+    if (wr_last < wr_first) { w_end = kv_begin; w_min_limit = kv_end; }   // warp has no valid rows
+    else {
+      w_end = min(kv_end, seg.p + wr_last / g.G + 1);
+      w_min_limit = min(kv_end, seg.p + wr_first / g.G + 1);
+    }
+  }
+
+  uint32_t qa[KS][4];
+  {
+    const uint16_t* q_lo = P.q + ((long long)(seg.q_off + qi_lo) * g.Hq + hd_lo) * D + 2 * (lane & 3);
+    const uint16_t* q_hi = P.q + ((long long)(seg.q_off + qi_hi) * g.Hq + hd_hi) * D + 2 * (lane & 3);
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qa[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(q_lo + ks * 16) : 0u;
+      qa[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(q_hi + ks * 16) : 0u;
+      qa[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(q_lo + ks * 16 + 8) : 0u;
+      qa[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(q_hi + ks * 16 + 8) : 0u;
+    }
+  }
+
+  float o[NT][4];
+#pragma unroll
+  for (int i = 0; i < NT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+  const float sl2 = P.scale_log2e;
+
+  for (int st = 0; st < n_st; ++st) {
+    const int slot = st % kStages;
+    mbar_wait(smem_u32(&s_full[slot]), (st / kStages) & 1, abort_flag, P.status);
+    const int key0 = kv_begin + st * kStageKeys;
+    const uint32_t stage = smem_base + slot * STAGE_BYTES;
+    const int kb_first = DECODE ? warp : 0;
+    const int step_key0 = key0 + kb_first * 16;
+    if (step_key0 < w_end) {
+      const int nkb = min(STEP_KB, (w_end - step_key0 + 15) >> 4);
+      float s[STEP_KB * 2][4];
+#pragma unroll
+      for (int b = 0; b < STEP_KB; ++b) {
+        if (b < nkb) {
+          const int koff = (kb_first + b) * 16;            // key offset inside the stage
+          const uint32_t pbase = stage + (koff / g.S) * g.head_bytes;
+          const int row0 = koff % g.S;
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            float(&acc)[4] = s[b * 2 + nt];
+            acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+            const int slot_row = row0 + nt * 8 + (lane & 7);
+#pragma unroll
+            for (int k2 = 0; k2 < KS / 2; ++k2) {
+              uint32_t b0, b1, b2, b3;
+              ldsm_x4(pbase + blk_chunk_offset(g.S, slot_row, k2 * 4 + (lane >> 3)), b0, b1, b2, b3);
+              mma_bf16(acc, qa[2 * k2], b0, b1);
+              mma_bf16(acc, qa[2 * k2 + 1], b2, b3);
+            }
+          }
+        }
+      }
+      // ---- scale, mask, online softmax ----
+      const int step_end = step_key0 + nkb * 16;
+      const bool need_mask = step_end > w_min_limit;
+      float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+      for (int t = 0; t < STEP_KB * 2; ++t) {
+        if (t < nkb * 2) {
+          const int j = step_key0 + t * 8 + 2 * (lane & 3);
+          float t0 = s[t][0] * sl2, t1 = s[t][1] * sl2, t2 = s[t][2] * sl2, t3 = s[t][3] * sl2;
+          if (need_mask) {
+            if (j >= kv_limit_lo) t0 = -INFINITY;
+            if (j + 1 >= kv_limit_lo) t1 = -INFINITY;
+            if (j >= kv_limit_hi) t2 = -INFINITY;
+            if (j + 1 >= kv_limit_hi) t3 = -INFINITY;
+          }
+          s[t][0] = t0; s[t][1] = t1; s[t][2] = t2; s[t][3] = t3;
+          mx_lo = fmaxf(mx_lo, fmaxf(t0, t1));
+          mx_hi = fmaxf(mx_hi, fmaxf(t2, t3));
+        }
+      }
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+      const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+      const float mu_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, mu_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+      const float a_lo = fast_exp2(m_lo - mu_lo), a_hi = fast_exp2(m_hi - mu_hi);
+      m_lo = mn_lo; m_hi = mn_hi;
+      if (__any_sync(0xffffffffu, a_lo != 1.f || a_hi != 1.f)) {
+#pragma unroll
+        for (int i = 0; i < NT; ++i) { o[i][0] *= a_lo; o[i][1] *= a_lo; o[i][2] *= a_hi; o[i][3] *= a_hi; }
+      }
+      float ps_lo = 0.f, ps_hi = 0.f;
+#pragma unroll
+      for (int t = 0; t < STEP_KB * 2; ++t) {
+        if (t < nkb * 2) {
+          s[t][0] = fast_exp2(s[t][0] - mu_lo); s[t][1] = fast_exp2(s[t][1] - mu_lo);
+          s[t][2] = fast_exp2(s[t][2] - mu_hi); s[t][3] = fast_exp2(s[t][3] - mu_hi);
+          ps_lo += s[t][0] + s[t][1];
+          ps_hi += s[t][2] + s[t][3];
+        }
+      }
+      l_lo = l_lo * a_lo + ps_lo;
+      l_hi = l_hi * a_hi + ps_hi;
+      // ---- O += P.V ----
+#pragma unroll
+      for (int b = 0; b < STEP_KB; ++b) {
+        if (b < nkb) {
+          const int koff = (kb_first + b) * 16;
+          const uint32_t vbase = stage + (koff / g.S) * g.head_bytes + g.kblock_bytes;
+          const int row0 = koff % g.S;
+          const int blk_key0 = key0 + koff;
+          if (blk_key0 + 16 > kv_end) {
+            // slots past the end of the item hold whatever the page held before: clear V there so that
+            // weight 0 times stale bits cannot produce NaN
+            const int first = kv_end - blk_key0;           // 1..15
+            uint8_t* vgen = smem_gen + (vbase - smem_base);
+            for (int idx = lane; idx < (16 - first) * (D / 8); idx += 32) {
+              const int rr = row0 + first + idx / (D / 8), c = idx % (D / 8);
+              *reinterpret_cast<uint4*>(vgen + blk_chunk_offset(g.S, rr, c)) = make_uint4(0, 0, 0, 0);
+            }
+            __syncwarp();
+          }
+          uint32_t pa[4];
+          pa[0] = pack_bf16(s[2 * b][0], s[2 * b][1]);
+          pa[1] = pack_bf16(s[2 * b][2], s[2 * b][3]);
+          pa[2] = pack_bf16(s[2 * b + 1][0], s[2 * b + 1][1]);
+          pa[3] = pack_bf16(s[2 * b + 1][2], s[2 * b + 1][3]);
+          const int vrow = row0 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+          for (int n2 = 0; n2 < NT / 2; ++n2) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4_t(vbase + blk_chunk_offset(g.S, vrow, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
+            mma_bf16(o[2 * n2], pa, b0, b1);
+            mma_bf16(o[2 * n2 + 1], pa, b2, b3);
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+  }
+
+  // ---- epilogue ----
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+  if (!DECODE) {
+    const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
+    const float e_lo = l_lo > 0.f ? m_lo + log2f(l_lo) : -INFINITY;
+    const float e_hi = l_hi > 0.f ? m_hi + log2f(l_hi) : -INFINITY;
+    const int dcol = 2 * (lane & 3);
+    if (direct) {
+      const long long o_lo = ((long long)(seg.q_off + qi_lo) * g.Hq + hd_lo), o_hi = ((long long)(seg.q_off + qi_hi) * g.Hq + hd_hi);
+#pragma unroll
+      for (int i = 0; i < NT; ++i) {
+        if (v_lo) *reinterpret_cast<uint32_t*>(P.out + o_lo * D + i * 8 + dcol) = pack_bf16(o[i][0] * inv_lo, o[i][1] * inv_lo);
+        if (v_hi) *reinterpret_cast<uint32_t*>(P.out + o_hi * D + i * 8 + dcol) = pack_bf16(o[i][2] * inv_hi, o[i][3] * inv_hi);
+      }
+      if (P.lse != nullptr && (lane & 3) == 0) {
+        if (v_lo) P.lse[o_lo] = e_lo * kLn2;
+        if (v_hi) P.lse[o_hi] = e_hi * kLn2;
+      }
+    } else {
+      const long long p_lo = seg.part_base + (long long)(split * seg.n + qi_lo) * g.Hq + hd_lo;
+      const long long p_hi = seg.part_base + (long long)(split * seg.n + qi_hi) * g.Hq + hd_hi;
+#pragma unroll
+      for (int i = 0; i < NT; ++i) {
+        if (v_lo) *reinterpret_cast<float2*>(P.part_o + p_lo * D + i * 8 + dcol) = make_float2(o[i][0] * inv_lo, o[i][1] * inv_lo);
+        if (v_hi) *reinterpret_cast<float2*>(P.part_o + p_hi * D + i * 8 + dcol) = make_float2(o[i][2] * inv_hi, o[i][3] * inv_hi);
+      }
+      if ((lane & 3) == 0) {
+        if (v_lo) P.part_lse[p_lo] = e_lo;
+        if (v_hi) P.part_lse[p_hi] = e_hi;
+      }
+    }
+    return;
+  }
+
+  // DECODE: the four warps hold partial (m, l, O) over disjoint keys of the same 16 rows; combine through
+  // shared memory (the stage ring is free: every copy that was issued has been consumed).
+  named_bar_sync(1, kConsumerWarps * 32);
+  float* s_o = reinterpret_cast<float*>(smem_gen);                    // [warp][16][D]
+  float* s_m = s_o + kConsumerWarps * 16 * D;                         // [warp][16]
+  float* s_l = s_m + kConsumerWarps * 16;
+  {
+    float* wo = s_o + warp * 16 * D;
+    const int rl = lane >> 2, dcol = 2 * (lane & 3);
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+      *reinterpret_cast<float2*>(wo + rl * D + i * 8 + dcol) = make_float2(o[i][0], o[i][1]);
+      *reinterpret_cast<float2*>(wo + (rl + 8) * D + i * 8 + dcol) = make_float2(o[i][2], o[i][3]);
+    }
+    if ((lane & 3) == 0) {
+      s_m[warp * 16 + rl] = m_lo; s_m[warp * 16 + rl + 8] = m_hi;
+      s_l[warp * 16 + rl] = l_lo; s_l[warp * 16 + rl + 8] = l_hi;
+    }
+  }
+  named_bar_sync(1, kConsumerWarps * 32);
+  {
+    constexpr int DSEG = D / 8;               // 128 threads = 16 rows x 8 column segments
+    const int t = threadIdx.x;
+    const int rr = t >> 3, d0 = (t & 7) * DSEG;
+    const int r = tile_row0 + rr;
+    if (r < R) {
+      float mw[kConsumerWarps], mstar = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) { mw[w] = s_m[w * 16 + rr]; mstar = fmaxf(mstar, mw[w]); }
+      const float mu = (mstar == -INFINITY) ? 0.f : mstar;
+      float f[kConsumerWarps], lstar = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) { f[w] = fast_exp2(mw[w] - mu); lstar += f[w] * s_l[w * 16 + rr]; }
+      const float inv = lstar > 0.f ? 1.f / lstar : 0.f;
+      const float e2 = lstar > 0.f ? mstar + log2f(lstar) : -INFINITY;
+      const int qi = r / g.G, hd = kvh * g.G + (r - qi * g.G);
+      float acc[DSEG];
+#pragma unroll
+      for (int d = 0; d < DSEG; ++d) {
+        float a = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) a += f[w] * s_o[(w * 16 + rr) * D + d0 + d];
+        acc[d] = a * inv;
+      }
+      if (direct) {
+        const long long orow = (long long)(seg.q_off + qi) * g.Hq + hd;
+        uint32_t* dst = reinterpret_cast<uint32_t*>(P.out + orow * D + d0);
+#pragma unroll
+        for (int d = 0; d < DSEG; d += 2) dst[d >> 1] = pack_bf16(acc[d], acc[d + 1]);
+        if (P.lse != nullptr && (t & 7) == 0) P.lse[orow] = e2 * kLn2;
+      } else {
+        const long long prow = seg.part_base + (long long)(split * seg.n + qi) * g.Hq + hd;
+        float* dst = P.part_o + prow * D + d0;
+#pragma unroll
+        for (int d = 0; d < DSEG; d += 4) *reinterpret_cast<float4*>(dst + d) = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
+        if ((t & 7) == 0) P.part_lse[prow] = e2;
+      }
+    }
+  }
+}
+
+cudaError_t attend_kernels_init() {
+  cudaError_t e;
+  e = cudaFuncSetAttribute(attend_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<128>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<128>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<64>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<64>::kSmemBytes);
+  return e;
+}
+
+cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s) {
+  if (p.n_items <= 0) return cudaSuccess;
+  if (p.g.D == 128) attend_mma_kernel<128, true><<<p.n_items, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
+  else attend_mma_kernel<64, true><<<p.n_items, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s) {
+  if (p.n_items <= 0) return cudaSuccess;
+  if (p.g.D == 128) attend_mma_kernel<128, false><<<p.n_items, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
+  else attend_mma_kernel<64, false><<<p.n_items, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Log-sum-exp merge of the split partials: one warp per (token, head) row.
+//   LSE = log2 sum_i 2^{LSE_i},  O = sum_i 2^{LSE_i - LSE} O_i;  fixed order, no atomics.
+__global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= P.n_rows) return;
+  const int si = find_segment(P.n_segs, row, [&](int i) { return P.segs[i].merge_base; });
+  const Segment seg = P.segs[si];
+  const int local = row - seg.merge_base;                 // token * Hq + head inside the segment
+  const long long stride = (long long)seg.n * P.Hq;       // partial rows per split
+  const long long p0 = seg.part_base + local;
+  float mstar = -INFINITY;
+  for (int s = 0; s < seg.n_splits; ++s) mstar = fmaxf(mstar, P.part_lse[p0 + s * stride]);
+  const float mu = (mstar == -INFINITY) ? 0.f : mstar;
+  const int per = P.D / 32;                               // 2 or 4 floats per lane
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float tot = 0.f;
+  for (int s = 0; s < seg.n_splits; ++s) {
+    const float e = P.part_lse[p0 + s * stride];
+    if (e == -INFINITY) continue;
+    const float w = exp2f(e - mu);
+    tot += w;
+    const float* po = P.part_o + (p0 + s * stride) * P.D + lane * per;
+    if (per == 4) {
+      const float4 v = *reinterpret_cast<const float4*>(po);
+      acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+    } else {
+      const float2 v = *reinterpret_cast<const float2*>(po);
+      acc[0] += w * v.x; acc[1] += w * v.y;
+    }
+  }
+  const float inv = tot > 0.f ? 1.f / tot : 0.f;
+  const long long orow = (long long)seg.q_off * P.Hq + local;
+  uint16_t* dst = P.out + orow * P.D + lane * per;
+  if (per == 4) {
+    uint2 v;
+    v.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+    v.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+    *reinterpret_cast<uint2*>(dst) = v;
+  } else {
+    *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0] * inv, acc[1] * inv);
+  }
+  if (P.lse != nullptr && lane == 0) P.lse[orow] = (tot > 0.f ? mstar + log2f(tot) : -INFINITY) * 0.6931471805599453f;
+}
+
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t s) {
+  if (p.n_rows <= 0) return cudaSuccess;
+  const int blocks = (p.n_rows + 7) / 8;
+  merge_kernel<<<blocks, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace tide

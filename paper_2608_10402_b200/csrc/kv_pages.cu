@@ -1,0 +1,109 @@
+// Page-append scatter, page-table delta update and logical read-back.
+//
+// Append is the GPU half of resuming a task under Continuous Task Batching (paper Section 4): the
+// observation tokens' K/V rows are copied into the task's pages next to its preserved state, which
+// replaces re-running prefill over the history (Section 1, first challenge).  It is a pure bit copy,
+// bound by HBM bandwidth: 2 * Hkv * D * 2 bytes read and as many written per new token.
+#include "tide_internal.h"
+
+namespace tide {
+
+__global__ void table_update_kernel(int32_t* __restrict__ table, const int32_t* __restrict__ idx,
+                                    const int32_t* __restrict__ val, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) table[idx[i]] = val[i];
+}
+
+cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  table_update_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, idx, val, n);
+  return cudaGetLastError();
+}
+
+// Byte offset of 16-byte chunk `c` (c = d / 8) of slot `slot` inside a K or V block.
+__device__ __forceinline__ int chunk_offset(int S, int slot, int c) {
+  return (c >> 3) * (S * 128) + slot * 128 + (((c & 7) ^ (slot & 7)) << 4);
+}
+
+constexpr int kAppendThreads = 256;
+constexpr int kAppendMaxRecsSmem = 1024;
+
+// One thread per 16-byte chunk of the source rows.  Chunks of a token are ordered [K|V][kv_head][c], so a
+// warp reads 512 contiguous source bytes and writes four full 128-byte lines.
+__global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const AppendParams P) {
+  __shared__ int32_t s_tok0[kAppendMaxRecsSmem];
+  const int n_recs = P.n_recs;
+  const bool in_smem = n_recs <= kAppendMaxRecsSmem;
+  if (in_smem) {
+    for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = P.recs[i].tok0;
+    __syncthreads();
+  }
+  const int cpr = P.g.D >> 3;                 // chunks per (token, head) row
+  const int cpt = 2 * P.g.Hkv * cpr;          // chunks per token, K and V
+  const long long total = (long long)P.n_tokens * cpt;
+  for (long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x; gid < total;
+       gid += (long long)gridDim.x * blockDim.x) {
+    const int tok = (int)(gid / cpt);
+    int rem = (int)(gid - (long long)tok * cpt);
+    const int kv = rem / (P.g.Hkv * cpr);
+    rem -= kv * P.g.Hkv * cpr;
+    const int h = rem / cpr;
+    const int c = rem - h * cpr;
+    int r;
+    if (in_smem) r = find_segment(n_recs, tok, [&](int i) { return s_tok0[i]; });
+    else r = find_segment(n_recs, tok, [&](int i) { return P.recs[i].tok0; });
+    const AppendRec rec = P.recs[r];
+    const int pos = rec.pos0 + (tok - rec.tok0);
+    const int lp = pos / P.g.S, slot = pos - lp * P.g.S;
+    const long long page = P.table[rec.table_off + lp];
+    const uint16_t* src = (kv ? P.new_v : P.new_k) + ((long long)tok * P.g.Hkv + h) * P.g.D + c * 8;
+    uint8_t* dst = P.pool + page * P.g.page_bytes + (long long)h * P.g.head_bytes + kv * P.g.kblock_bytes +
+                   chunk_offset(P.g.S, slot, c);
+    *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+  }
+}
+
+cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
+  if (p.n_tokens <= 0) return cudaSuccess;
+  const long long total = (long long)p.n_tokens * 2 * p.g.Hkv * (p.g.D / 8);
+  long long blocks = (total + kAppendThreads - 1) / kAppendThreads;
+  const long long cap = 148LL * 8 * 16;  // grid-stride beyond this
+  if (blocks > cap) blocks = cap;
+  append_scatter_kernel<<<(unsigned)blocks, kAppendThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+// Logical content of one task -> contiguous [len, Hkv, D]; inverse of the scatter above.
+__global__ void read_gather_kernel(const uint8_t* __restrict__ pool, const int32_t* __restrict__ table_row, int len,
+                                   uint16_t* __restrict__ out_k, uint16_t* __restrict__ out_v, const Geom g) {
+  const int cpr = g.D >> 3;
+  const int cpt = 2 * g.Hkv * cpr;
+  const long long total = (long long)len * cpt;
+  for (long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x; gid < total;
+       gid += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(gid / cpt);
+    int rem = (int)(gid - (long long)pos * cpt);
+    const int kv = rem / (g.Hkv * cpr);
+    rem -= kv * g.Hkv * cpr;
+    const int h = rem / cpr;
+    const int c = rem - h * cpr;
+    const int lp = pos / g.S, slot = pos - lp * g.S;
+    const long long page = table_row[lp];
+    const uint8_t* src = pool + page * g.page_bytes + (long long)h * g.head_bytes + kv * g.kblock_bytes +
+                         chunk_offset(g.S, slot, c);
+    uint16_t* dst = (kv ? out_v : out_k) + ((long long)pos * g.Hkv + h) * g.D + c * 8;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int len, uint16_t* out_k, uint16_t* out_v,
+                        const Geom& g, cudaStream_t s) {
+  if (len <= 0) return cudaSuccess;
+  const long long total = (long long)len * 2 * g.Hkv * (g.D / 8);
+  long long blocks = (total + 255) / 256;
+  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  read_gather_kernel<<<(unsigned)blocks, 256, 0, s>>>(pool, table_row, len, out_k, out_v, g);
+  return cudaGetLastError();
+}
+
+}  // namespace tide

@@ -1,0 +1,653 @@
+// Host side of libtide.so: the C ABI, the page allocator and per-task tables, the work planner and the
+// kernel launches.  See include/tide.h for the contract of every entry point.
+//
+// Allocator rule (what makes page tables reproducible): free pages are a LIFO stack primed so that a
+// fresh pool hands out free_order[0], free_order[1], ...; an append walks its tasks in array order and
+// pops one page each time a token lands on slot 0 of a new logical page; release and truncate push pages
+// back last-to-first.  Every call validates completely before it changes anything.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "tide_internal.h"
+
+using namespace tide;
+
+namespace {
+
+constexpr int kSlots = 4;                    // staging ring depth
+constexpr size_t kSlotPageIds = 64 * 1024;   // most new page ids per upload
+constexpr int kSlotRecs = 2048;              // most append records per upload
+constexpr int kTargetItemsPerSm = 8;
+constexpr int kNumSms = 148;
+constexpr long long kPartRowsBase = 256 * 1024;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  size_t off_status, off_table, off_meta, off_part_o, off_part_lse, off_stage_k, off_stage_v, off_stage_q,
+      off_stage_out, off_stage_lse, total;
+  size_t slot_bytes;
+  long long part_rows;
+};
+
+struct Slot {
+  uint8_t* host = nullptr;
+  uint8_t* dev = nullptr;
+  cudaEvent_t ev = nullptr;
+  bool used = false;
+};
+
+}  // namespace
+
+struct tide_kv {
+  tide_kv_config_t cfg;
+  Geom g;
+  Layout lay;
+  int device = 0;
+  uint8_t* pool = nullptr;
+  uint8_t* ws = nullptr;
+  int32_t* d_table = nullptr;
+  int* d_status = nullptr;
+  float* d_part_o = nullptr;
+  float* d_part_lse = nullptr;
+  Slot slots[kSlots];
+  int next_slot = 0;
+  int* h_status = nullptr;  // pinned
+  // bookkeeping
+  std::vector<int32_t> free_stack;  // back() is the next page handed out
+  std::vector<uint8_t> live;
+  std::vector<int32_t> len;
+  std::vector<std::vector<int32_t>> pages;
+  std::vector<int32_t> mark;  // scratch for duplicate detection
+  int32_t mark_gen = 0;
+  int64_t used_tokens = 0;
+  // last plan
+  int64_t last_decode_items = 0, last_prefill_items = 0, last_merge_rows = 0, last_launches = 0;
+  int64_t append_launches = 0;
+};
+
+namespace {
+
+bool valid_geometry(const tide_kv_config_t* c) {
+  if (c == nullptr) return false;
+  if (c->num_layers != 1) return false;
+  if (c->num_kv_heads <= 0 || c->num_q_heads <= 0 || c->num_q_heads % c->num_kv_heads != 0) return false;
+  if (c->num_q_heads / c->num_kv_heads > 16) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->page_size != 16 && c->page_size != 32) return false;
+  if (c->max_tasks <= 0 || c->max_pages_per_task <= 0 || c->max_batch_rows <= 0) return false;
+  if (c->num_pages <= 0 || c->num_pages > 0x7fffffffLL || c->max_batch_tokens <= 0) return false;
+  if ((long long)c->max_tasks * c->max_pages_per_task > 0x7fffffffLL) return false;
+  if (c->max_batch_tokens * (long long)c->num_q_heads > 0x7fffffffLL) return false;
+  return true;
+}
+
+Geom make_geom(const tide_kv_config_t* c) {
+  Geom g;
+  g.Hq = c->num_q_heads; g.Hkv = c->num_kv_heads; g.D = c->head_dim; g.S = c->page_size; g.G = g.Hq / g.Hkv;
+  g.max_pages_per_task = c->max_pages_per_task;
+  g.kblock_bytes = g.D * g.S * 2;
+  g.head_bytes = 2 * g.kblock_bytes;
+  g.page_bytes = (long long)g.head_bytes * g.Hkv;
+  return g;
+}
+
+Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
+  Layout L;
+  size_t off = 0;
+  L.off_status = off; off += 256;
+  L.off_table = off; off = align_up(off + (size_t)c->max_tasks * c->max_pages_per_task * 4, 256);
+  L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 +
+                              (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
+  L.off_meta = off; off += L.slot_bytes * kSlots;
+  L.part_rows = kPartRowsBase + (long long)g.Hq * c->max_batch_rows * 4;
+  L.off_part_o = off; off = align_up(off + (size_t)L.part_rows * g.D * 4, 256);
+  L.off_part_lse = off; off = align_up(off + (size_t)L.part_rows * 4, 256);
+  const size_t kv_rows = (size_t)c->max_batch_tokens * g.Hkv * g.D * 2;
+  const size_t q_rows = (size_t)c->max_batch_tokens * g.Hq * g.D * 2;
+  L.off_stage_k = off; off = align_up(off + kv_rows, 256);
+  L.off_stage_v = off; off = align_up(off + kv_rows, 256);
+  L.off_stage_q = off; off = align_up(off + q_rows, 256);
+  L.off_stage_out = off; off = align_up(off + q_rows, 256);
+  L.off_stage_lse = off; off = align_up(off + (size_t)c->max_batch_tokens * g.Hq * 4, 256);
+  L.total = off;
+  return L;
+}
+
+bool is_permutation(const int32_t* order, int64_t n, std::vector<uint8_t>& seen) {
+  seen.assign((size_t)n, 0);
+  for (int64_t i = 0; i < n; ++i) {
+    const int32_t p = order[i];
+    if (p < 0 || p >= n || seen[(size_t)p]) return false;
+    seen[(size_t)p] = 1;
+  }
+  return true;
+}
+
+void prime_free_stack(tide_kv* kv, const int32_t* order) {
+  const int64_t n = kv->cfg.num_pages;
+  kv->free_stack.resize((size_t)n);
+  for (int64_t i = 0; i < n; ++i) kv->free_stack[(size_t)(n - 1 - i)] = order ? order[i] : (int32_t)i;
+}
+
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+bool task_in_range(const tide_kv* kv, int32_t t) { return t >= 0 && t < kv->cfg.max_tasks; }
+
+// Takes the next staging slot, waiting until the device work that last used it has finished.
+int acquire_slot(tide_kv* kv, Slot** out) {
+  Slot& s = kv->slots[kv->next_slot];
+  kv->next_slot = (kv->next_slot + 1) % kSlots;
+  if (s.used && cudaEventSynchronize(s.ev) != cudaSuccess) return TIDE_ERR_CUDA;
+  *out = &s;
+  return TIDE_OK;
+}
+
+int release_slot(Slot* s, cudaStream_t st) {
+  s->used = true;
+  return cudaEventRecord(s->ev, st) == cudaSuccess ? TIDE_OK : TIDE_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tide_strerror(int code) {
+  switch (code) {
+    case TIDE_OK: return "ok";
+    case TIDE_ERR_INVALID_ARG: return "invalid argument";
+    case TIDE_ERR_UNKNOWN_TASK: return "unknown task";
+    case TIDE_ERR_TASK_EXISTS: return "task already exists";
+    case TIDE_ERR_DUPLICATE_TASK: return "task named twice in one append";
+    case TIDE_ERR_NO_PAGES: return "not enough free pages";
+    case TIDE_ERR_TABLE_FULL: return "task would exceed max_pages_per_task";
+    case TIDE_ERR_CTX_RANGE: return "row violates 1 <= q_len <= ctx_len <= resident length";
+    case TIDE_ERR_WORKSPACE: return "pool, workspace or batch limit too small";
+    case TIDE_ERR_CUDA: return "CUDA runtime error";
+    case TIDE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    default: return "unknown tide status";
+  }
+}
+
+int tide_kv_required_bytes(const tide_kv_config_t* cfg, size_t* pool_bytes, size_t* workspace_bytes) {
+  if (!valid_geometry(cfg)) return TIDE_ERR_INVALID_ARG;
+  const Geom g = make_geom(cfg);
+  if (pool_bytes) *pool_bytes = (size_t)cfg->num_pages * (size_t)g.page_bytes;
+  if (workspace_bytes) *workspace_bytes = make_layout(cfg, g).total;
+  return TIDE_OK;
+}
+
+int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
+  if (out == nullptr || !valid_geometry(cfg)) return TIDE_ERR_INVALID_ARG;
+  if (cfg->pool == nullptr || cfg->workspace == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (((uintptr_t)cfg->pool & 1023) || ((uintptr_t)cfg->workspace & 255)) return TIDE_ERR_INVALID_ARG;
+  const Geom g = make_geom(cfg);
+  const Layout lay = make_layout(cfg, g);
+  if (cfg->pool_bytes < (size_t)cfg->num_pages * (size_t)g.page_bytes || cfg->workspace_bytes < lay.total)
+    return TIDE_ERR_WORKSPACE;
+  std::vector<uint8_t> seen;
+  if (cfg->free_order && !is_permutation(cfg->free_order, cfg->num_pages, seen)) return TIDE_ERR_INVALID_ARG;
+
+  tide_kv* kv = new (std::nothrow) tide_kv();
+  if (!kv) return TIDE_ERR_INVALID_ARG;
+  kv->cfg = *cfg;
+  kv->cfg.free_order = nullptr;
+  kv->g = g;
+  kv->lay = lay;
+  kv->pool = (uint8_t*)cfg->pool;
+  kv->ws = (uint8_t*)cfg->workspace;
+  kv->d_status = (int*)(kv->ws + lay.off_status);
+  kv->d_table = (int32_t*)(kv->ws + lay.off_table);
+  kv->d_part_o = (float*)(kv->ws + lay.off_part_o);
+  kv->d_part_lse = (float*)(kv->ws + lay.off_part_lse);
+  bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
+  ok = ok && attend_kernels_init() == cudaSuccess;
+  ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
+  ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
+  for (int i = 0; ok && i < kSlots; ++i) {
+    ok = cudaHostAlloc((void**)&kv->slots[i].host, lay.slot_bytes, cudaHostAllocDefault) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&kv->slots[i].ev, cudaEventDisableTiming) == cudaSuccess;
+    kv->slots[i].dev = kv->ws + lay.off_meta + (size_t)i * lay.slot_bytes;
+  }
+  if (!ok) {
+    tide_kv_destroy(kv);
+    return TIDE_ERR_CUDA;
+  }
+  kv->live.assign((size_t)cfg->max_tasks, 0);
+  kv->len.assign((size_t)cfg->max_tasks, 0);
+  kv->pages.resize((size_t)cfg->max_tasks);
+  kv->mark.assign((size_t)cfg->max_tasks, 0);
+  prime_free_stack(kv, cfg->free_order);
+  *out = kv;
+  return TIDE_OK;
+}
+
+int tide_kv_destroy(tide_kv_t* kv) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  for (int i = 0; i < kSlots; ++i) {
+    if (kv->slots[i].host) cudaFreeHost(kv->slots[i].host);
+    if (kv->slots[i].ev) cudaEventDestroy(kv->slots[i].ev);
+  }
+  if (kv->h_status) cudaFreeHost(kv->h_status);
+  delete kv;
+  return TIDE_OK;
+}
+
+int tide_kv_reset(tide_kv_t* kv, const int32_t* free_order) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  std::vector<uint8_t> seen;
+  if (free_order && !is_permutation(free_order, kv->cfg.num_pages, seen)) return TIDE_ERR_INVALID_ARG;
+  std::fill(kv->live.begin(), kv->live.end(), 0);
+  std::fill(kv->len.begin(), kv->len.end(), 0);
+  for (auto& p : kv->pages) p.clear();
+  kv->used_tokens = 0;
+  prime_free_stack(kv, free_order);
+  return TIDE_OK;
+}
+
+int tide_kv_alloc(tide_kv_t* kv, int32_t task, int64_t reserve_tokens) {
+  if (kv == nullptr || !task_in_range(kv, task) || reserve_tokens < 0) return TIDE_ERR_INVALID_ARG;
+  if (kv->live[task]) return TIDE_ERR_TASK_EXISTS;
+  if ((int64_t)kv->free_stack.size() * kv->g.S < reserve_tokens) return TIDE_ERR_NO_PAGES;
+  kv->live[task] = 1;
+  kv->len[task] = 0;
+  kv->pages[task].clear();
+  return TIDE_OK;
+}
+
+int tide_kv_release(tide_kv_t* kv, int32_t task) {
+  if (kv == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  auto& pg = kv->pages[task];
+  for (size_t i = pg.size(); i-- > 0;) kv->free_stack.push_back(pg[i]);
+  pg.clear();
+  kv->used_tokens -= kv->len[task];
+  kv->len[task] = 0;
+  kv->live[task] = 0;
+  return TIDE_OK;
+}
+
+int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len) {
+  if (kv == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  if (new_len < 0 || new_len > kv->len[task]) return TIDE_ERR_INVALID_ARG;
+  auto& pg = kv->pages[task];
+  const size_t keep = (size_t)ceil_div(new_len, kv->g.S);
+  while (pg.size() > keep) {
+    kv->free_stack.push_back(pg.back());
+    pg.pop_back();
+  }
+  kv->used_tokens -= kv->len[task] - new_len;
+  kv->len[task] = new_len;
+  return TIDE_OK;
+}
+
+int tide_kv_task_len(tide_kv_t* kv, int32_t task, int32_t* len) {
+  if (kv == nullptr || len == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  *len = kv->len[task];
+  return TIDE_OK;
+}
+
+int tide_kv_page_table(tide_kv_t* kv, int32_t task, int32_t* out, int32_t cap, int32_t* n_pages) {
+  if (kv == nullptr || n_pages == nullptr || !task_in_range(kv, task) || cap < 0) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  const auto& pg = kv->pages[task];
+  *n_pages = (int32_t)pg.size();
+  if (out != nullptr) {
+    if ((size_t)cap < pg.size()) return TIDE_ERR_INVALID_ARG;
+    std::memcpy(out, pg.data(), pg.size() * sizeof(int32_t));
+  }
+  return TIDE_OK;
+}
+
+int tide_kv_usage(tide_kv_t* kv, int64_t* used_tokens, int64_t* free_pages) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (used_tokens) *used_tokens = kv->used_tokens;
+  if (free_pages) *free_pages = (int64_t)kv->free_stack.size();
+  return TIDE_OK;
+}
+
+int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr,
+                   const void* new_k, const void* new_v, void* stream) {
+  if (kv == nullptr || layer != 0 || n_tasks < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_tasks == 0) return TIDE_OK;
+  if (task_ids == nullptr || indptr == nullptr || indptr[0] != 0) return TIDE_ERR_INVALID_ARG;
+  const Geom& g = kv->g;
+  for (int j = 0; j < n_tasks; ++j)
+    if (indptr[j + 1] < indptr[j]) return TIDE_ERR_INVALID_ARG;
+  for (int j = 0; j < n_tasks; ++j) {
+    if (!task_in_range(kv, task_ids[j])) return TIDE_ERR_INVALID_ARG;
+    if (!kv->live[task_ids[j]]) return TIDE_ERR_UNKNOWN_TASK;
+  }
+  if (++kv->mark_gen == 0x7fffffff) {
+    std::fill(kv->mark.begin(), kv->mark.end(), 0);
+    kv->mark_gen = 1;
+  }
+  for (int j = 0; j < n_tasks; ++j) {
+    if (kv->mark[task_ids[j]] == kv->mark_gen) return TIDE_ERR_DUPLICATE_TASK;
+    kv->mark[task_ids[j]] = kv->mark_gen;
+  }
+  const int T = indptr[n_tasks];
+  if (T > 0 && (new_k == nullptr || new_v == nullptr || ((uintptr_t)new_k & 15) || ((uintptr_t)new_v & 15)))
+    return TIDE_ERR_INVALID_ARG;
+  long long need = 0;
+  for (int j = 0; j < n_tasks; ++j) {
+    const int t = task_ids[j], c = indptr[j + 1] - indptr[j];
+    if ((long long)kv->len[t] + c > 0x7fffffffLL) return TIDE_ERR_TABLE_FULL;
+    const int after = ceil_div(kv->len[t] + c, g.S);
+    if (after > g.max_pages_per_task) return TIDE_ERR_TABLE_FULL;
+    need += after - ceil_div(kv->len[t], g.S);
+  }
+  if (need > (long long)kv->free_stack.size()) return TIDE_ERR_NO_PAGES;
+
+  // ---- mutation: host tables first, then upload the deltas and scatter, in bounded batches ----
+  cudaStream_t st = (cudaStream_t)stream;
+  kv->append_launches = 0;
+  int j = 0, done_in_task = 0;  // progress cursor: task index, tokens of that task already recorded
+  int rc = TIDE_OK;
+  while (j < n_tasks) {
+    Slot* slot;
+    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+    AppendRec* recs = (AppendRec*)(slot->host + 256);
+    int32_t* idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
+    int32_t* val = idx + kSlotPageIds;
+    int n_recs = 0;
+    size_t n_ids = 0;
+    int tok_lo = -1, tok_hi = -1;
+    while (j < n_tasks && n_recs < kSlotRecs) {
+      const int t = task_ids[j];
+      const int c = indptr[j + 1] - indptr[j];
+      int remaining = c - done_in_task;
+      if (remaining == 0) { ++j; done_in_task = 0; continue; }
+      const int pos0 = kv->len[t];
+      // tokens that fit: up to the page-id budget of this upload
+      const int room_in_last = (int)((long long)ceil_div(pos0, g.S) * g.S - pos0);
+      const size_t ids_left = kSlotPageIds - n_ids;
+      long long can = room_in_last + (long long)ids_left * g.S;
+      if (can <= 0) break;
+      const int take = (int)std::min<long long>(remaining, can);
+      const int new_pages = ceil_div(pos0 + take, g.S) - ceil_div(pos0, g.S);
+      auto& pg = kv->pages[t];
+      for (int k = 0; k < new_pages; ++k) {
+        const int32_t page = kv->free_stack.back();
+        kv->free_stack.pop_back();
+        idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size();
+        val[n_ids] = page;
+        ++n_ids;
+        pg.push_back(page);
+      }
+      AppendRec& r = recs[n_recs++];
+      r.table_off = t * g.max_pages_per_task;
+      r.pos0 = pos0;
+      r.tok0 = indptr[j] + done_in_task;
+      r.count = take;
+      if (tok_lo < 0) tok_lo = r.tok0;
+      tok_hi = r.tok0 + take;
+      kv->len[t] += take;
+      kv->used_tokens += take;
+      done_in_task += take;
+      if (done_in_task == c) { ++j; done_in_task = 0; }
+      if (n_ids == kSlotPageIds) break;
+    }
+    if (n_recs == 0) continue;
+    // records hold absolute token indices; the kernel is launched over [tok_lo, tok_hi)
+    for (int k = 0; k < n_recs; ++k) recs[k].tok0 -= tok_lo;
+    const size_t up_bytes = 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
+    // only the used prefixes of the three arrays need to travel
+    if (cudaMemcpyAsync(slot->dev + 256, slot->host + 256, (size_t)n_recs * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return TIDE_ERR_CUDA;
+    if (n_ids > 0) {
+      uint8_t* didx = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec);
+      if (cudaMemcpyAsync(didx, idx, n_ids * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (cudaMemcpyAsync(didx + kSlotPageIds * 4, val, n_ids * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (launch_table_update(kv->d_table, (const int32_t*)didx, (const int32_t*)(didx + kSlotPageIds * 4), (int)n_ids, st) != cudaSuccess)
+        return TIDE_ERR_CUDA;
+      ++kv->append_launches;
+    }
+    (void)up_bytes;
+    AppendParams ap;
+    ap.pool = kv->pool;
+    ap.table = kv->d_table;
+    ap.recs = (const AppendRec*)(slot->dev + 256);
+    ap.n_recs = n_recs;
+    ap.n_tokens = tok_hi - tok_lo;
+    ap.new_k = (const uint16_t*)new_k + (size_t)tok_lo * g.Hkv * g.D;
+    ap.new_v = (const uint16_t*)new_v + (size_t)tok_lo * g.Hkv * g.D;
+    ap.g = g;
+    if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++kv->append_launches;
+    if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+  }
+  return TIDE_OK;
+}
+
+int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k, void* out_v, void* stream) {
+  if (kv == nullptr || layer != 0 || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  if (kv->len[task] == 0) return TIDE_OK;
+  if (out_k == nullptr || out_v == nullptr || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15)) return TIDE_ERR_INVALID_ARG;
+  const int32_t* row = kv->d_table + (size_t)task * kv->g.max_pages_per_task;
+  if (launch_read(kv->pool, row, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
+    return TIDE_ERR_CUDA;
+  return TIDE_OK;
+}
+
+int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows, const int32_t* page_table,
+                const void* q, float scale, void* out, float* lse, void* stream) {
+  if (kv == nullptr || layer != 0 || n_rows < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_rows == 0) return TIDE_OK;
+  if (rows == nullptr || q == nullptr || out == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)lse & 3) || ((uintptr_t)page_table & 3)) return TIDE_ERR_INVALID_ARG;
+  if (!(scale == scale) || n_rows > kv->cfg.max_batch_rows) return n_rows > kv->cfg.max_batch_rows ? TIDE_ERR_WORKSPACE : TIDE_ERR_INVALID_ARG;
+  const Geom& g = kv->g;
+  long long total_q = 0;
+  for (int b = 0; b < n_rows; ++b) {
+    const tide_row_t& r = rows[b];
+    if (!task_in_range(kv, r.task)) return TIDE_ERR_INVALID_ARG;
+    if (!kv->live[r.task]) return TIDE_ERR_UNKNOWN_TASK;
+    if (!(r.q_len >= 1 && r.q_len <= r.ctx_len && r.ctx_len <= kv->len[r.task])) return TIDE_ERR_CTX_RANGE;
+    total_q += r.q_len;
+  }
+  if (total_q > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
+
+  // ---- plan: one segment per row, decode-style (<= 16 packed rows) or tile-style ----
+  struct RowPlan { int b; bool decode; int n_mtiles; long long items; };
+  std::vector<RowPlan> plan((size_t)n_rows);
+  long long w_dec = 0, w_tile = 0, items_tile_nosplit = 0;
+  {
+    for (int b = 0; b < n_rows; ++b) {
+      const tide_row_t& r = rows[b];
+      const int R = r.q_len * g.G;
+      RowPlan& p = plan[(size_t)b];
+      p.b = b;
+      p.decode = R <= kDecodeTileRows;
+      p.n_mtiles = p.decode ? 1 : ceil_div(R, kMmaTileRows);
+      p.items = (long long)g.Hkv * p.n_mtiles;
+      if (p.decode) w_dec += (long long)g.Hkv * r.ctx_len;
+      else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
+    }
+  }
+  const long long target = (long long)kNumSms * kTargetItemsPerSm;
+  long long chunk_dec = std::max<long long>(256, align_up((size_t)(w_dec / target + 1), kStageKeys));
+  long long chunk_tile = (items_tile_nosplit >= target / 2)
+                             ? (1LL << 30)
+                             : std::max<long long>(2048, align_up((size_t)(w_tile / target + 1), kStageKeys));
+  std::vector<Segment> seg_dec, seg_tile, seg_merge;
+  long long items_dec = 0, items_tile = 0, part_rows = 0, merge_rows = 0;
+  for (int attempt = 0; attempt < 40; ++attempt) {
+    seg_dec.clear(); seg_tile.clear();
+    part_rows = 0;
+    long long qoff = 0;
+    for (int b = 0; b < n_rows; ++b) {
+      const tide_row_t& r = rows[b];
+      const RowPlan& p = plan[(size_t)b];
+      const long long chunk_target = p.decode ? chunk_dec : chunk_tile;
+      int n_splits = (int)std::min<long long>(kMaxSplits, ((long long)r.ctx_len + chunk_target - 1) / chunk_target);
+      n_splits = std::max(1, n_splits);
+      int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), kStageKeys);
+      n_splits = ceil_div(r.ctx_len, chunk);
+      Segment s{};
+      s.table_off = r.task * g.max_pages_per_task;
+      s.q_off = (int32_t)qoff;
+      s.n = r.q_len;
+      s.p = r.ctx_len - r.q_len;
+      s.n_mtiles = p.n_mtiles;
+      s.n_splits = n_splits;
+      s.chunk = chunk;
+      s.part_base = 0;
+      if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
+      (p.decode ? seg_dec : seg_tile).push_back(s);
+      qoff += r.q_len;
+    }
+    if (part_rows <= kv->lay.part_rows) break;
+    chunk_dec *= 2;
+    chunk_tile = std::min<long long>(chunk_tile * 2, 1LL << 30);
+    if (attempt == 39) return TIDE_ERR_WORKSPACE;
+  }
+  // heaviest items first, so the tail of the grid is made of short items
+  auto heavier = [](const Segment& a, const Segment& b) {
+    return std::min(a.chunk, a.p + a.n) > std::min(b.chunk, b.p + b.n);
+  };
+  std::stable_sort(seg_dec.begin(), seg_dec.end(), heavier);
+  std::stable_sort(seg_tile.begin(), seg_tile.end(), heavier);
+  long long part_cursor = 0;
+  for (auto* v : {&seg_dec, &seg_tile}) {
+    long long base = 0;
+    for (Segment& s : *v) {
+      s.item_base = (int32_t)base;
+      base += (long long)g.Hkv * s.n_mtiles * s.n_splits;
+      if (base > 0x7fffffffLL) return TIDE_ERR_WORKSPACE;
+      if (s.n_splits > 1) {
+        s.part_base = (int32_t)part_cursor;
+        part_cursor += (long long)s.n_splits * s.n * g.Hq;
+        s.merge_base = (int32_t)merge_rows;
+        merge_rows += (long long)s.n * g.Hq;
+        seg_merge.push_back(s);
+      }
+    }
+    (v == &seg_dec ? items_dec : items_tile) = base;
+  }
+  const size_t n_all = seg_dec.size() + seg_tile.size() + seg_merge.size();
+  if (n_all * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  Slot* slot;
+  int rc;
+  if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+  Segment* h = (Segment*)(slot->host + 256);
+  std::copy(seg_dec.begin(), seg_dec.end(), h);
+  std::copy(seg_tile.begin(), seg_tile.end(), h + seg_dec.size());
+  std::copy(seg_merge.begin(), seg_merge.end(), h + seg_dec.size() + seg_tile.size());
+  if (cudaMemcpyAsync(slot->dev + 256, h, n_all * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  const Segment* d = (const Segment*)(slot->dev + 256);
+
+  AttendParams ap;
+  ap.pool = kv->pool;
+  ap.table = page_table ? page_table : kv->d_table;
+  ap.q = (const uint16_t*)q;
+  ap.out = (uint16_t*)out;
+  ap.lse = lse;
+  ap.part_o = kv->d_part_o;
+  ap.part_lse = kv->d_part_lse;
+  ap.scale_log2e = scale * 1.4426950408889634f;
+  ap.status = kv->d_status;
+  ap.g = g;
+  int64_t launches = 0;
+  if (items_dec > 0) {
+    ap.segs = d; ap.n_segs = (int)seg_dec.size(); ap.n_items = (int)items_dec;
+    if (launch_attend_decode(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++launches;
+  }
+  if (items_tile > 0) {
+    ap.segs = d + seg_dec.size(); ap.n_segs = (int)seg_tile.size(); ap.n_items = (int)items_tile;
+    if (launch_attend_tile(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++launches;
+  }
+  if (merge_rows > 0) {
+    MergeParams mp;
+    mp.segs = d + seg_dec.size() + seg_tile.size();
+    mp.n_segs = (int)seg_merge.size();
+    mp.n_rows = (int)merge_rows;
+    mp.part_o = kv->d_part_o; mp.part_lse = kv->d_part_lse;
+    mp.out = (uint16_t*)out; mp.lse = lse; mp.Hq = g.Hq; mp.D = g.D;
+    if (launch_merge(mp, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++launches;
+  }
+  if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+  kv->last_decode_items = items_dec;
+  kv->last_prefill_items = items_tile;
+  kv->last_merge_rows = merge_rows;
+  kv->last_launches = launches + kv->append_launches;
+  kv->append_launches = 0;
+  return TIDE_OK;
+}
+
+int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows, const void* new_k,
+                   const void* new_v, const void* q, float scale, void* out, float* lse, void* stream) {
+  if (kv == nullptr || layer != 0 || n_rows < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_rows == 0) return TIDE_OK;
+  if (rows == nullptr || new_k == nullptr || new_v == nullptr || q == nullptr || out == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (n_rows > kv->cfg.max_batch_rows) return TIDE_ERR_WORKSPACE;
+  const Geom& g = kv->g;
+  std::vector<int32_t> ids((size_t)n_rows), indptr((size_t)n_rows + 1);
+  indptr[0] = 0;
+  for (int b = 0; b < n_rows; ++b) {
+    const tide_row_t& r = rows[b];
+    if (!task_in_range(kv, r.task)) return TIDE_ERR_INVALID_ARG;
+    if (!kv->live[r.task]) return TIDE_ERR_UNKNOWN_TASK;
+    if (r.q_len < 1 || (long long)kv->len[r.task] + r.q_len != r.ctx_len) return TIDE_ERR_CTX_RANGE;
+    ids[(size_t)b] = r.task;
+    if ((long long)indptr[(size_t)b] + r.q_len > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
+    indptr[(size_t)b + 1] = indptr[(size_t)b] + r.q_len;
+  }
+  const size_t T = (size_t)indptr[(size_t)n_rows];
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* dk = kv->ws + kv->lay.off_stage_k;
+  uint8_t* dv = kv->ws + kv->lay.off_stage_v;
+  uint8_t* dq = kv->ws + kv->lay.off_stage_q;
+  uint8_t* dout = kv->ws + kv->lay.off_stage_out;
+  float* dlse = (float*)(kv->ws + kv->lay.off_stage_lse);
+  const size_t kv_bytes = T * g.Hkv * g.D * 2, q_bytes = T * g.Hq * g.D * 2;
+  // validate the append (duplicates, pages) BEFORE any copy by running it first: it is all-or-nothing
+  if (cudaMemcpyAsync(dk, new_k, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (cudaMemcpyAsync(dv, new_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  int rc = tide_kv_append(kv, layer, n_rows, ids.data(), indptr.data(), dk, dv, stream);
+  if (rc != TIDE_OK) return rc;
+  rc = tide_attend(kv, layer, n_rows, rows, nullptr, dq, scale, dout, lse ? dlse : nullptr, stream);
+  if (rc != TIDE_OK) return rc;
+  if (cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (lse && cudaMemcpyAsync(lse, dlse, T * g.Hq * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
+  return TIDE_OK;
+}
+
+int tide_status(tide_kv_t* kv, void* stream) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(kv->h_status, kv->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
+  const int code = *kv->h_status;
+  if (code != 0) {
+    if (cudaMemsetAsync(kv->d_status, 0, sizeof(int), st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  return code == 0 ? TIDE_OK : code;
+}
+
+int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,
+                   int64_t* kernel_launches) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (decode_items) *decode_items = kv->last_decode_items;
+  if (prefill_items) *prefill_items = kv->last_prefill_items;
+  if (merge_rows) *merge_rows = kv->last_merge_rows;
+  if (kernel_launches) *kernel_launches = kv->last_launches;
+  return TIDE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+// Internal declarations shared by the host code and the kernels of libtide.so.
+//
+// Physical page layout (private; callers see logical content only):
+//   pool[page][kv_head][K|V][slab = d/64][slot][64 bf16]
+// i.e. for one (page, kv_head) the K block and then the V block, each block made of D/64 slabs of
+// S rows x 128 bytes.  Inside every group of 8 rows the 16-byte chunk c of row r is stored at chunk
+// position c ^ (r & 7) (the 128-byte swizzle of the tensor-core shared-memory layouts).  A plain
+// contiguous bulk copy of a block therefore lands in shared memory ready both for conflict-free
+// ldmatrix and for tcgen05 matrix descriptors, with no tensor map.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/tide.h"
+
+namespace tide {
+
+constexpr int kStageKeys = 64;       // keys per pipeline stage of the mma.sync attention kernel
+constexpr int kMaxSplits = 128;      // most KV splits of one row
+constexpr int kDecodeTileRows = 16;  // packed (query, head) rows per decode-style work item
+constexpr int kMmaTileRows = 64;     // packed rows per work item of the warp-MMA tile path
+constexpr int kUmmaTileRows = 128;   // packed rows per work item of the tcgen05 path
+constexpr long long kWaitLimitNs = 2000000000LL;  // bound of every in-kernel wait
+
+struct Geom {
+  int Hq, Hkv, D, S, G;
+  int max_pages_per_task;
+  int kblock_bytes;  // one K (or V) block of a (page, head): D*S*2
+  int head_bytes;    // K block + V block
+  long long page_bytes;
+};
+
+// One batch row as the kernels see it.  Items of a segment are numbered
+// ((kv_head * n_splits) + split) * n_mtiles + m_tile from item_base.
+struct __align__(16) Segment {
+  int32_t table_off;   // task * max_pages_per_task
+  int32_t q_off;       // index of the row's first query token in q / out
+  int32_t n;           // q_len
+  int32_t p;           // preserved prefix = ctx_len - q_len
+  int32_t item_base;
+  int32_t n_mtiles;
+  int32_t n_splits;
+  int32_t chunk;       // keys per split, a multiple of kStageKeys
+  int32_t part_base;   // first partial row ((split * n + token) * Hq + head) when n_splits > 1
+  int32_t merge_base;  // first row of this segment in the merge launch
+  int32_t pad0, pad1;
+};
+static_assert(sizeof(Segment) == 48, "Segment layout");
+
+struct AttendParams {
+  const uint8_t* pool;
+  const int32_t* table;
+  const Segment* segs;
+  int n_segs;
+  int n_items;
+  const uint16_t* q;
+  uint16_t* out;
+  float* lse;        // may be null
+  float* part_o;     // [partial rows][D] fp32, normalised
+  float* part_lse;   // [partial rows] fp32, base-2 log units
+  float scale_log2e;
+  int* status;
+  Geom g;
+};
+
+struct MergeParams {
+  const Segment* segs;
+  int n_segs;
+  int n_rows;
+  const float* part_o;
+  const float* part_lse;
+  uint16_t* out;
+  float* lse;
+  int Hq, D;
+};
+
+struct __align__(16) AppendRec {
+  int32_t table_off;  // task * max_pages_per_task
+  int32_t pos0;       // position in the task of the record's first token
+  int32_t tok0;       // index of that token in new_k / new_v
+  int32_t count;
+};
+
+struct AppendParams {
+  uint8_t* pool;
+  const int32_t* table;
+  const AppendRec* recs;
+  int n_recs;
+  int n_tokens;
+  const uint16_t* new_k;
+  const uint16_t* new_v;
+  Geom g;
+};
+
+cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s);
+cudaError_t launch_append(const AppendParams& p, cudaStream_t s);
+cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int len, uint16_t* out_k, uint16_t* out_v,
+                        const Geom& g, cudaStream_t s);
+cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s);
+cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s);
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);
+cudaError_t attend_kernels_init();
+
+#ifdef __CUDACC__
+// ---------------------------------------------------------------------------------------------
+// device helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ long long global_ns() {
+  long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  `abort_flag` lives in shared memory: once any thread of the CTA has given up, every
+// later wait returns at once so that the CTA still walks its normal control flow to the end.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  if (*abort_flag) return false;
+  const long long t0 = global_ns();
+  int spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 255) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, (int)TIDE_ERR_DEVICE_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+// 1-D bulk copy global -> shared, completion counted on an mbarrier.  16-byte aligned, size % 16 == 0.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// D[16x8] += A[16x16] * B[16x8], bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Locate the segment that owns work index `idx` (segments sorted by the base returned by `base_of`).
+template <typename F>
+__device__ __forceinline__ int find_segment(int n_segs, int idx, F base_of) {
+  int lo = 0, hi = n_segs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (base_of(mid) <= idx) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+#endif  // __CUDACC__
+
+}  // namespace tide

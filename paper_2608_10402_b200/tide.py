@@ -1,0 +1,211 @@
+"""ctypes binding of libtide.so: the same names as include/tide.h, argument marshalling only.
+
+Every step of the path runs inside the CUDA library; this module only turns torch tensors / numpy
+arrays into pointers.  There is no fallback: if libtide.so is missing or cannot be loaded the import
+of this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtide.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNKNOWN_TASK, ERR_TASK_EXISTS, ERR_DUPLICATE_TASK = -1, -2, -3, -4
+ERR_NO_PAGES, ERR_TABLE_FULL, ERR_CTX_RANGE, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = -5, -6, -7, -8, -9, -10
+
+
+class TideError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+class tide_row_t(ctypes.Structure):
+    _fields_ = [("task", ctypes.c_int32), ("q_len", ctypes.c_int32), ("ctx_len", ctypes.c_int32)]
+
+
+class tide_kv_config_t(ctypes.Structure):
+    _fields_ = [
+        ("num_layers", ctypes.c_int32), ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32), ("max_tasks", ctypes.c_int32),
+        ("max_pages_per_task", ctypes.c_int32), ("max_batch_rows", ctypes.c_int32),
+        ("num_pages", ctypes.c_int64), ("max_batch_tokens", ctypes.c_int64),
+        ("pool", ctypes.c_void_p), ("pool_bytes", ctypes.c_size_t),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("free_order", ctypes.c_void_p),
+    ]
+
+
+EXPORTS = [
+    "tide_strerror", "tide_kv_required_bytes", "tide_kv_create", "tide_kv_destroy", "tide_kv_reset",
+    "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
+    "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
+]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_10402_b200.build` "
+                      "(there is no fallback path)")
+lib = ctypes.CDLL(LIB_PATH)
+lib.tide_strerror.restype = ctypes.c_char_p
+lib.tide_strerror.argtypes = [ctypes.c_int]
+for _name in EXPORTS[1:]:
+    getattr(lib, _name).restype = ctypes.c_int
+
+
+def strerror(code: int) -> str:
+    return lib.tide_strerror(int(code)).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise TideError(code, what)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _ptr(x):
+    """Device / host pointer of a torch tensor, numpy array, int or None."""
+    if x is None:
+        return ctypes.c_void_p(0)
+    if isinstance(x, int):
+        return ctypes.c_void_p(x)
+    if isinstance(x, np.ndarray):
+        return ctypes.c_void_p(x.ctypes.data)
+    return ctypes.c_void_p(x.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def rows_array(rows):
+    """[(task, q_len, ctx_len)] -> ctypes array of tide_row_t."""
+    arr = (tide_row_t * len(rows))()
+    for i, (t, n, c) in enumerate(rows):
+        arr[i].task, arr[i].q_len, arr[i].ctx_len = int(t), int(n), int(c)
+    return arr
+
+
+def make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens):
+    cfg = tide_kv_config_t()
+    cfg.num_layers = 1
+    cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.page_size = int(Hq), int(Hkv), int(D), int(S)
+    cfg.max_tasks, cfg.max_pages_per_task, cfg.max_batch_rows = int(max_tasks), int(max_pages_per_task), int(max_batch_rows)
+    cfg.num_pages, cfg.max_batch_tokens = int(num_pages), int(max_batch_tokens)
+    return cfg
+
+
+def tide_kv_required_bytes(cfg):
+    pb, wb = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib.tide_kv_required_bytes(ctypes.byref(cfg), ctypes.byref(pb), ctypes.byref(wb)), "tide_kv_required_bytes")
+    return pb.value, wb.value
+
+
+class TideKV:
+    """One paged cache on the current CUDA device.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens,
+                 free_order=None, device="cuda"):
+        import torch
+        self.cfg = make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens)
+        pb, wb = tide_kv_required_bytes(self.cfg)
+        # PyTorch only supplies device memory (and streams)
+        self.pool = torch.empty(pb + 1024, dtype=torch.uint8, device=device)
+        self.workspace = torch.empty(wb + 256, dtype=torch.uint8, device=device)
+        pool_ptr = (self.pool.data_ptr() + 1023) // 1024 * 1024
+        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.cfg.pool, self.cfg.pool_bytes = pool_ptr, pb
+        self.cfg.workspace, self.cfg.workspace_bytes = ws_ptr, wb
+        self._free_order = None if free_order is None else _i32(free_order)
+        self.cfg.free_order = None if free_order is None else self._free_order.ctypes.data
+        self.Hq, self.Hkv, self.D, self.S = int(Hq), int(Hkv), int(D), int(S)
+        self.handle = ctypes.c_void_p(0)
+        _check(lib.tide_kv_create(ctypes.byref(self.cfg), ctypes.byref(self.handle)), "tide_kv_create")
+
+    def close(self):
+        if self.handle:
+            lib.tide_kv_destroy(self.handle)
+            self.handle = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- lifecycle ----
+    def reset(self, free_order=None):
+        fo = None if free_order is None else _i32(free_order)
+        _check(lib.tide_kv_reset(self.handle, _ptr(fo)), "tide_kv_reset")
+
+    def alloc(self, task, reserve_tokens=0):
+        _check(lib.tide_kv_alloc(self.handle, ctypes.c_int32(task), ctypes.c_int64(reserve_tokens)), "tide_kv_alloc")
+
+    def release(self, task):
+        _check(lib.tide_kv_release(self.handle, ctypes.c_int32(task)), "tide_kv_release")
+
+    def truncate(self, task, new_len):
+        _check(lib.tide_kv_truncate(self.handle, ctypes.c_int32(task), ctypes.c_int32(new_len)), "tide_kv_truncate")
+
+    def append(self, task_ids, indptr, new_k, new_v, stream=None):
+        ids, ip = _i32(task_ids), _i32(indptr)
+        assert ip.shape[0] == ids.shape[0] + 1
+        _check(lib.tide_kv_append(self.handle, ctypes.c_int32(0), ctypes.c_int32(ids.shape[0]), _ptr(ids), _ptr(ip),
+                                  _ptr(new_k), _ptr(new_v), _stream(stream)), "tide_kv_append")
+
+    def attend(self, rows, q, scale, out, lse=None, page_table=None, stream=None):
+        arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
+        _check(lib.tide_attend(self.handle, ctypes.c_int32(0), ctypes.c_int32(len(arr)), arr, _ptr(page_table), _ptr(q),
+                               ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)), "tide_attend")
+
+    def step_host(self, rows, new_k, new_v, q, scale, out, lse=None, stream=None):
+        arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
+        _check(lib.tide_step_host(self.handle, ctypes.c_int32(0), ctypes.c_int32(len(arr)), arr, _ptr(new_k), _ptr(new_v),
+                                  _ptr(q), ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)), "tide_step_host")
+
+    # ---- introspection ----
+    def task_len(self, task):
+        v = ctypes.c_int32(0)
+        _check(lib.tide_kv_task_len(self.handle, ctypes.c_int32(task), ctypes.byref(v)), "tide_kv_task_len")
+        return v.value
+
+    def page_table(self, task):
+        n = ctypes.c_int32(0)
+        _check(lib.tide_kv_page_table(self.handle, ctypes.c_int32(task), None, ctypes.c_int32(0), ctypes.byref(n)), "tide_kv_page_table")
+        out = np.empty(n.value, dtype=np.int32)
+        _check(lib.tide_kv_page_table(self.handle, ctypes.c_int32(task), _ptr(out), ctypes.c_int32(n.value), ctypes.byref(n)), "tide_kv_page_table")
+        return out
+
+    def usage(self):
+        u, f = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib.tide_kv_usage(self.handle, ctypes.byref(u), ctypes.byref(f)), "tide_kv_usage")
+        return u.value, f.value
+
+    def read(self, task, stream=None):
+        """Logical K, V of a task as torch uint16-bit tensors (int16 view) [len, Hkv, D] on the device."""
+        import torch
+        L = self.task_len(task)
+        k = torch.empty((L, self.Hkv, self.D), dtype=torch.int16, device=self.pool.device)
+        v = torch.empty_like(k)
+        _check(lib.tide_kv_read(self.handle, ctypes.c_int32(0), ctypes.c_int32(task), _ptr(k), _ptr(v), _stream(stream)), "tide_kv_read")
+        return k, v
+
+    def status(self, stream=None):
+        return lib.tide_status(self.handle, _stream(stream))
+
+    def last_plan(self):
+        a, b, c, d = (ctypes.c_int64(0) for _ in range(4))
+        _check(lib.tide_last_plan(self.handle, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(d)), "tide_last_plan")
+        return {"decode_items": a.value, "prefill_items": b.value, "merge_rows": c.value, "kernel_launches": d.value}
