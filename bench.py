@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of one CTB step (page append + mixed-batch attention) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+A step = tide_kv_append of every row's new tokens + tide_attend of the whole batch, on a synthetic batch
+shaped like the paper's workloads (see paper_2608_10402_b200/inputs.py).  Prints ONE JSON line.
+`value` is the KV-read rate of the decode rows inside the mixed step (their KV bytes / the device time of
+the decode-style kernel in that step); `append_prefill_tflops` is the other half of the metric (flops of
+the resume rows / device time of the tile kernel).  Multi-GPU runs are independent replicas (tasks never
+move between ranks), launched with torch.distributed.run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "mixed resume batch: KV-read GB/s vs HBM peak; append-prefill TFLOP/s vs peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------------------
+def build_state(w, torch, tide, seed):
+    """Cache with every task's preserved prefix resident, plus this step's device inputs."""
+    total_q = int(w.n_new.sum())
+    kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task,
+                     max_batch_rows=w.B, max_batch_tokens=total_q, free_order=w.free_order)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    for b in range(w.B):
+        kv.alloc(int(w.task[b]))
+    for b in range(w.B):
+        p = int(w.prefix[b])
+        k = torch.randn((p, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+        v = torch.randn((p, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+        kv.append([int(w.task[b])], [0, p], k, v)
+    torch.cuda.synchronize()
+    sig = torch.ones((total_q, 1, 1), device="cuda")
+    off = 0
+    for b in range(w.B):            # image tokens of a multimodal chunk: K/V ~ N(0, 1.5)
+        ni = int(w.n_image[b])
+        if ni:
+            sig[off:off + ni] = w.image_sigma
+        off += int(w.n_new[b])
+    new_k = (torch.randn((total_q, w.Hkv, w.D), device="cuda", generator=gen) * sig).to(torch.bfloat16)
+    new_v = (torch.randn((total_q, w.Hkv, w.D), device="cuda", generator=gen) * sig).to(torch.bfloat16)
+    q = torch.randn((total_q, w.Hq, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    lse = torch.empty((total_q, w.Hq), device="cuda", dtype=torch.float32)
+    return kv, new_k, new_v, q, out, lse
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_10402_b200 import inputs, tide
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+
+    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank)
+    kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank)
+    rows = tide.rows_array(w.rows())
+    ids = np.asarray(w.task, dtype=np.int32)
+    indptr = np.concatenate([[0], np.cumsum(w.n_new)]).astype(np.int32)
+    order_back = [(int(w.task[b]), int(w.prefix[b])) for b in reversed(range(w.B))]
+
+    def step():
+        kv.append(ids, indptr, new_k, new_v)
+        kv.attend(rows, q, w.scale, out, lse)
+
+    def rollback():
+        for t, p in order_back:       # host only: every task back to its prefix, pages return in LIFO order
+            kv.truncate(t, p)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+        rollback()
+    assert kv.status() == tide.OK
+    launches_per_step = kv.last_plan()["kernel_launches"]
+    plan = kv.last_plan()
+
+    # ---- timed region 1: K whole steps, device time ----
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+        rollback()
+    ev1.record()
+    barrier()
+    step_ms = ev0.elapsed_time(ev1) / args.steps
+
+    # ---- timed region 2: the same steps with per-phase events (append / decode kernel / tile kernel / merge) ----
+    kv.set_profiling(True)
+    phases = {"append": [], "decode": [], "tile": [], "merge": []}
+    for _ in range(args.steps):
+        step()
+        ph = kv.phase_ms()
+        rollback()
+        for k in phases:
+            phases[k].append(ph[k])
+    kv.set_profiling(False)
+    clocks = sampler.stop()
+    ph_ms = {k: float(np.mean(v)) for k, v in phases.items()}
+    assert kv.status() == tide.OK
+
+    # ---- timed region 3: end to end from pinned HOST buffers through tide_step_host ----
+    hk, hv, hq = new_k.cpu().pin_memory(), new_v.cpu().pin_memory(), q.cpu().pin_memory()
+    hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    hlse = torch.empty(lse.shape, dtype=lse.dtype).pin_memory()
+    for _ in range(2):
+        kv.step_host(rows, hk, hv, hq, w.scale, hout, hlse)
+        rollback()
+    barrier()
+    e2e_steps = max(1, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        kv.step_host(rows, hk, hv, hq, w.scale, hout, hlse)
+        rollback()
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+
+    # ---- numbers ----
+    dec_bytes = w.decode_kv_bytes()
+    res_flops = w.resume_flops()
+    t = torch.tensor([step_ms, ph_ms["decode"], ph_ms["tile"], ph_ms["append"], ph_ms["merge"], e2e_ms],
+                     device="cuda", dtype=torch.float64)
+    tot = torch.tensor([dec_bytes, res_flops], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    step_ms, dec_ms, tile_ms, app_ms, mrg_ms, e2e_ms = [float(x) for x in t.tolist()]
+    dec_bytes_all, res_flops_all = [float(x) for x in tot.tolist()]
+    kv_gbs = dec_bytes_all / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
+    tflops = res_flops_all / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0
+
+    if rank == 0:
+        n_app = int(w.n_new.sum())
+        app_bytes = 2 * w.kv_bytes_per_token() * n_app
+        use_tensor = res_flops > 0 and tile_ms >= dec_ms
+        sustained = step_ms * args.steps > 1000.0
+        tpeak = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+        roof_tensor = {"bound": "tensor", "kernel": "attend tile kernel (resume rows)",
+                       "achieved": res_flops / (ph_ms["tile"] * 1e-3) / 1e12 if ph_ms["tile"] > 0 else 0.0,
+                       "peak": tpeak, "unit": "TFLOP/s", "traffic": None,
+                       "peak_source": f"{peaks['_source']} ({'sustained' if sustained else 'burst'} bf16)"}
+        roof_tensor["frac"] = roof_tensor["achieved"] / tpeak
+        roof_hbm = {"bound": "hbm", "kernel": "attend decode kernel (decode rows)",
+                    "achieved": dec_bytes / (ph_ms["decode"] * 1e-3) / 1e9 if ph_ms["decode"] > 0 else 0.0,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "traffic": None, "peak_source": f"{peaks['_source']} (copy)"}
+        roof_hbm["frac"] = roof_hbm["achieved"] / peaks["hbm_gbs"]
+        line = {
+            "metric": METRIC, "value": kv_gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "append_prefill_tflops": tflops,
+            "phase_ms": {"append": app_ms, "decode_kernel": dec_ms, "tile_kernel": tile_ms, "merge": mrg_ms},
+            "append_gbs": app_bytes / (ph_ms["append"] * 1e-3) / 1e9 if ph_ms["append"] > 0 else 0.0,
+            "config": {"workload": f"configs[{args.config - 1}]: {w.name}", "tasks": w.B,
+                       "decode_rows": int((w.n_new == 1).sum()), "resume_rows": int((w.n_new > 1).sum()),
+                       "new_tokens": n_app, "prefix_tokens": int(w.prefix.sum()),
+                       "heads": f"{w.Hq}q/{w.Hkv}kv", "head_dim": w.D, "page_size": w.S,
+                       "decode_kv_bytes": dec_bytes, "resume_flops": res_flops,
+                       "l2": "inputs larger than L2 (no flush)" if dec_bytes + app_bytes > 2 * 126e6 else "smaller than L2",
+                       "parallelism": f"replicas x{world}", "plan": plan},
+            "roofline": roof_tensor if use_tensor else roof_hbm,
+            "roofline_decode": roof_hbm, "roofline_prefill": roof_tensor,
+            "e2e": {"value": dec_bytes_all / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+                    "definition": "decode-row KV bytes / whole host-buffer step (H2D new K,V,Q + append + attend + D2H out,lse)",
+                    "h2d_bytes_per_step": int(hk.numel() * 2 * 2 + hq.numel() * 2),
+                    "d2h_bytes_per_step": int(hout.numel() * 2 + hlse.numel() * 4)},
+            "gpu_launches": int(launches_per_step * args.steps),
+            "clocks": clocks,
+        }
+        line["cpu_baseline"] = cpu_baseline(args.config, budget_s=args.cpu_budget)
+        print(json.dumps(line))
+    kv.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------------------
+def _oracle_sample(config, n_decode=6, n_resume_q=24):
+    """A bounded sample of the workload for the CPU oracle: a few decode rows and a few queries of one
+    resume row, with their whole contexts resident in an oracle cache."""
+    from oracle.paged_kv import PagedKVOracle
+    from paper_2608_10402_b200 import inputs
+    w = inputs.make_workload(config)
+    dec = [b for b in range(w.B) if w.n_new[b] == 1][:n_decode]
+    res = [b for b in range(w.B) if w.n_new[b] > 1][:1]
+    picked = dec + res
+    pages = int(sum((int(w.ctx[b]) + w.S - 1) // w.S for b in picked)) + 4
+    c = PagedKVOracle(pages, w.S, w.Hkv, w.D, w.max_tasks, w.max_pages_per_task,
+                      free_order=np.random.default_rng(5).permutation(pages))
+    rows, qs, items = [], [], []
+    for r, b in enumerate(picked):
+        k, v = w.task_kv(b)
+        t = int(w.task[b])
+        c.alloc(t)
+        c.append([t], [0, k.shape[0]], k, v)
+        rows.append(w.rows()[b])
+        qs.append(w.task_q(b))
+        n = int(w.n_new[b])
+        if n == 1:
+            items.append((r, 0))
+        else:
+            items.extend((r, int(i)) for i in np.linspace(0, n - 1, n_resume_q).astype(int))
+    kv_bytes = sum(w.kv_bytes_per_token() * (rows[r][2] - rows[r][1] + i + 1) for r, i in items)
+    return w, c, rows, np.concatenate(qs), items, kv_bytes
+
+
+def cpu_baseline(config, budget_s=20.0):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    from oracle import cbuild
+    w, c, rows, q, items, kv_bytes = _oracle_sample(config)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        cbuild.attend_paged(c, rows, q, w.scale, items=items)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt > budget_s * 0.5 or reps >= 50:
+            break
+    return {"value": kv_bytes * reps / dt / 1e9, "unit": "GB/s", "cores": cbuild.threads(), "kind": "oracle",
+            "sample": f"{len(items)} (row, query) items of configs[{config - 1}] ({sum(1 for r in rows if r[1] == 1)} decode rows + "
+                      f"sampled queries of 1 resume row), KV bytes visible to each item / oracle seconds, {reps} passes",
+            "seconds": dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import cbuild
+    w, c, rows, q, items, kv_bytes = _oracle_sample(args.config)
+    for _ in range(max(1, min(args.warmup, 2))):
+        cbuild.attend_paged(c, rows, q, w.scale, items=items)
+    steps = max(1, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        cbuild.attend_paged(c, rows, q, w.scale, items=items)
+    dt = (time.perf_counter() - t0) / steps
+    val = kv_bytes / dt / 1e9
+    sample = f"each step = {len(items)} (row, query) items of configs[{args.config - 1}] through the float64 oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": max(1, min(args.warmup, 2)), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"configs[{args.config - 1}]: {w.name}", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cbuild.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, help="BASELINE.json configs[config-1]; default the mixed resume batch")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -154,6 +154,14 @@ int tide_status(tide_kv_t* kv, void* stream);
 int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,
                    int64_t* kernel_launches);
 
+/* Per-phase device timing of the calls that follow (CUDA events on the caller's stream; off by default).
+ * tide_phase_ms waits for the most recent tide_attend and returns the milliseconds spent in the most
+ * recent tide_kv_append (0 if none since the last query), in the decode-style attention kernel, in the
+ * tensor-tile attention kernel and in the merge kernel: the split of one mixed CTB step into its
+ * KV-bandwidth-bound and its tensor-bound halves. */
+int tide_set_profiling(tide_kv_t* kv, int enable);
+int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile_ms, float* merge_ms);
+
 const char* tide_strerror(int code);
 
 #ifdef __cplusplus

@@ -67,6 +67,11 @@ struct tide_kv {
   // last plan
   int64_t last_decode_items = 0, last_prefill_items = 0, last_merge_rows = 0, last_launches = 0;
   int64_t append_launches = 0;
+  // optional per-phase timing (events on the caller's stream)
+  bool profiling = false;
+  cudaEvent_t ev_append[2] = {nullptr, nullptr};
+  cudaEvent_t ev_attend[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool have_append_times = false, have_attend_times = false;
 };
 
 namespace {
@@ -233,6 +238,8 @@ int tide_kv_destroy(tide_kv_t* kv) {
     if (kv->slots[i].ev) cudaEventDestroy(kv->slots[i].ev);
   }
   if (kv->h_status) cudaFreeHost(kv->h_status);
+  for (cudaEvent_t e : kv->ev_append) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : kv->ev_attend) if (e) cudaEventDestroy(e);
   delete kv;
   return TIDE_OK;
 }
@@ -348,6 +355,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
   // ---- mutation: host tables first, then upload the deltas and scatter, in bounded batches ----
   cudaStream_t st = (cudaStream_t)stream;
   kv->append_launches = 0;
+  if (kv->profiling) cudaEventRecord(kv->ev_append[0], st);
   int j = 0, done_in_task = 0;  // progress cursor: task index, tokens of that task already recorded
   int rc = TIDE_OK;
   while (j < n_tasks) {
@@ -422,6 +430,10 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
     if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++kv->append_launches;
     if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+  }
+  if (kv->profiling) {
+    cudaEventRecord(kv->ev_append[1], st);
+    kv->have_append_times = true;
   }
   return TIDE_OK;
 }
@@ -558,16 +570,19 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   ap.status = kv->d_status;
   ap.g = g;
   int64_t launches = 0;
+  if (kv->profiling) cudaEventRecord(kv->ev_attend[0], st);
   if (items_dec > 0) {
     ap.segs = d; ap.n_segs = (int)seg_dec.size(); ap.n_items = (int)items_dec;
     if (launch_attend_decode(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
+  if (kv->profiling) cudaEventRecord(kv->ev_attend[1], st);
   if (items_tile > 0) {
     ap.segs = d + seg_dec.size(); ap.n_segs = (int)seg_tile.size(); ap.n_items = (int)items_tile;
     if (launch_attend_tile(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
+  if (kv->profiling) cudaEventRecord(kv->ev_attend[2], st);
   if (merge_rows > 0) {
     MergeParams mp;
     mp.segs = d + seg_dec.size() + seg_tile.size();
@@ -577,6 +592,10 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
     mp.out = (uint16_t*)out; mp.lse = lse; mp.Hq = g.Hq; mp.D = g.D;
     if (launch_merge(mp, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
+  }
+  if (kv->profiling) {
+    cudaEventRecord(kv->ev_attend[3], st);
+    kv->have_attend_times = true;
   }
   if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   kv->last_decode_items = items_dec;
@@ -638,6 +657,38 @@ int tide_status(tide_kv_t* kv, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
   }
   return code == 0 ? TIDE_OK : code;
+}
+
+int tide_set_profiling(tide_kv_t* kv, int enable) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (enable && kv->ev_append[0] == nullptr) {
+    for (cudaEvent_t& e : kv->ev_append) if (cudaEventCreate(&e) != cudaSuccess) return TIDE_ERR_CUDA;
+    for (cudaEvent_t& e : kv->ev_attend) if (cudaEventCreate(&e) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  kv->profiling = enable != 0;
+  kv->have_append_times = kv->have_attend_times = false;
+  return TIDE_OK;
+}
+
+int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile_ms, float* merge_ms) {
+  if (kv == nullptr || !kv->profiling) return TIDE_ERR_INVALID_ARG;
+  float a = 0.f, d = 0.f, t = 0.f, m = 0.f;
+  if (kv->have_append_times) {
+    if (cudaEventSynchronize(kv->ev_append[1]) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaEventElapsedTime(&a, kv->ev_append[0], kv->ev_append[1]) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  if (kv->have_attend_times) {
+    if (cudaEventSynchronize(kv->ev_attend[3]) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaEventElapsedTime(&d, kv->ev_attend[0], kv->ev_attend[1]) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaEventElapsedTime(&t, kv->ev_attend[1], kv->ev_attend[2]) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaEventElapsedTime(&m, kv->ev_attend[2], kv->ev_attend[3]) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  if (append_ms) *append_ms = a;
+  if (decode_ms) *decode_ms = d;
+  if (tile_ms) *tile_ms = t;
+  if (merge_ms) *merge_ms = m;
+  kv->have_append_times = false;
+  return TIDE_OK;
 }
 
 int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,

@@ -45,6 +45,7 @@ EXPORTS = [
     "tide_strerror", "tide_kv_required_bytes", "tide_kv_create", "tide_kv_destroy", "tide_kv_reset",
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
+    "tide_set_profiling", "tide_phase_ms",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -204,6 +205,14 @@ class TideKV:
 
     def status(self, stream=None):
         return lib.tide_status(self.handle, _stream(stream))
+
+    def set_profiling(self, enable):
+        _check(lib.tide_set_profiling(self.handle, ctypes.c_int(1 if enable else 0)), "tide_set_profiling")
+
+    def phase_ms(self):
+        v = [ctypes.c_float(0) for _ in range(4)]
+        _check(lib.tide_phase_ms(self.handle, *[ctypes.byref(x) for x in v]), "tide_phase_ms")
+        return {"append": v[0].value, "decode": v[1].value, "tile": v[2].value, "merge": v[3].value}
 
     def last_plan(self):
         a, b, c, d = (ctypes.c_int64(0) for _ in range(4))
