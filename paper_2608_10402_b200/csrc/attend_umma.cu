@@ -1,0 +1,443 @@
+// Append-prefill attention for resume rows on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// TMEM).
+//
+// What it computes (paper Section 4: a resumed task's appended observation tokens attend to the whole
+// preserved KV state instead of re-running prefill over the history): for a work item
+// (row, kv_head, m_tile, split), 256 packed rows r = q_index * G + g (two 128-row MMA tiles A and B) against
+// keys [kv_begin, kv_end), query q_index seeing keys [0, prefix + q_index]; online softmax in the base-2
+// domain; O and LSE written directly, or as normalised partials when the row is split over KV.
+// This is a dense contraction (n*G x ctx x D), so it is bound by the tensor pipe: 4*D flops per visible
+// (packed row, key) pair against Hkv*D*4 bytes per key shared by all packed rows.
+//
+// CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warp 8 streams K
+// and V tiles of 128 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
+// 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.
+//   S_t = Q_t . K_j^T   (SS MMA, 128x128x128, fp32 in TMEM)       t in {A, B}
+//   softmax WG t: TMEM -> registers, max / exp2 / sum, P_t as bf16 into shared memory
+//   O_t += P_t . V_j    (SS MMA, V tile used MN-major)
+// QK of tile j+1 is issued as soon as the softmax warpgroup has pulled S_t(j) into registers, so the tensor
+// pipe works on the other tile / the next keys while exponentials are computed.  O is only rescaled when a
+// row's running maximum grows by more than 2^8 (the final normalisation uses the same stale maximum, so the
+// result is exact); that happens on the first tiles only.
+// Every wait is bounded; a wait that runs out sets TIDE_ERR_DEVICE_TIMEOUT and the CTA drains and exits.
+#include <climits>
+
+#include "tide_internal.h"
+
+namespace tide {
+
+namespace umma {
+
+constexpr int D = 128;
+constexpr int kTileKeys = 128;
+constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA issuer, 2 idle warps}
+constexpr int kNumBuf = 3;                          // ring of K / V tiles: K0 V0 K1 V1 ...
+constexpr int kTileBytes = 128 * 128 * 2;           // one operand tile (Q half, P, K or V): 32 KB
+constexpr int kSlabBytes = 128 * 128;               // 128 rows x 128 bytes
+constexpr int kOffQ = 0;                            // Q_A, Q_B
+constexpr int kOffP = 2 * kTileBytes;               // P_A, P_B
+constexpr int kOffKV = 4 * kTileBytes;
+constexpr int kSmemBytes = (4 + kNumBuf) * kTileBytes + 1024;
+constexpr float kRescaleThreshold = 8.0f;           // log2 units
+
+// instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])),
+        "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])),
+        "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+struct Bars {
+  uint64_t kv_full[kNumBuf];
+  uint64_t kv_empty[kNumBuf];
+  uint64_t q_full;
+  uint64_t s_full[2];
+  uint64_t s_free[2];
+  uint64_t p_full[2];
+  uint64_t p_free[2];
+};
+
+__global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) Bars bars;
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Geom& g = P.g;
+
+  // ---- which item ----
+  const int item = blockIdx.x;
+  const int si = find_segment(P.n_segs, item, [&](int i) { return P.segs[i].item_base; });
+  const Segment seg = P.segs[si];
+  int local = item - seg.item_base;
+  const int m_tile = local % seg.n_mtiles;
+  local /= seg.n_mtiles;
+  const int split = local % seg.n_splits;
+  const int kvh = local / seg.n_splits;
+  const int R = seg.n * g.G;
+  const int item_row0 = m_tile * kUmmaTileRows * 2;
+  const int kv_begin = split * seg.chunk;
+  const bool direct = seg.n_splits == 1;
+  // per 128-row tile: rows present, last key any of its rows sees, number of 128-key tiles to process
+  int t_rows[2], t_end[2], t_tiles[2], t_min_limit[2];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r0 = item_row0 + t * 128;
+    t_rows[t] = max(0, min(128, R - r0));
+    if (t_rows[t] > 0) {
+      t_end[t] = min(kv_begin + seg.chunk, seg.p + (r0 + t_rows[t] - 1) / g.G + 1);
+      t_min_limit[t] = min(t_end[t], seg.p + r0 / g.G + 1);
+      t_tiles[t] = t_end[t] > kv_begin ? (t_end[t] - kv_begin + kTileKeys - 1) / kTileKeys : 0;
+    } else {
+      t_end[t] = kv_begin; t_min_limit[t] = kv_begin; t_tiles[t] = 0;
+    }
+  }
+  const int n_tiles = max(t_tiles[0], t_tiles[1]);
+  const int kv_end = max(t_end[0], t_end[1]);
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
+    mbar_init(smem_u32(&bars.q_full), 256);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&bars.s_full[t]), 1);
+      mbar_init(smem_u32(&bars.s_free[t]), 128);
+      mbar_init(smem_u32(&bars.p_full[t]), 128);
+      mbar_init(smem_u32(&bars.p_free[t]), 1);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem_base;
+  volatile int* abort_flag = &s_abort;
+
+  // register budget: the data-movement warpgroup gives registers to the two softmax warpgroups, which
+  // hold a whole 128-wide row of S per thread
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+  if (warp == 8) {
+    // ================= producer: K0 V0 K1 V1 ... into the ring =================
+    if (n_tiles > 0) {
+      const int pages_per_tile = kTileKeys / g.S;
+      const int slab_block = g.S * 128;                      // bytes of one slab of a page block
+      const int copies = pages_per_tile * 2;                 // (page, slab) pairs per operand tile
+      for (int idx = 0; idx < 2 * n_tiles; ++idx) {
+        const int buf = idx % kNumBuf, use = idx / kNumBuf;
+        if (use > 0) mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status);
+        const int j = idx >> 1, is_v = idx & 1;
+        const int key0 = kv_begin + j * kTileKeys;
+        const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
+        const uint32_t bar = smem_u32(&bars.kv_full[buf]);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * 2 * slab_block));
+        __syncwarp();
+        for (int c = lane; c < copies; c += 32) {
+          const int pg = c >> 1, slab = c & 1;
+          if (pg < npages) {
+            const long long page = P.table[seg.table_off + key0 / g.S + pg];
+            const uint8_t* src = P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes + is_v * g.kblock_bytes + slab * slab_block;
+            bulk_g2s(smem_base + kOffKV + buf * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
+          }
+        }
+      }
+      if (*abort_flag && lane == 0) {
+        for (int idx = max(0, 2 * n_tiles - kNumBuf); idx < 2 * n_tiles; ++idx) {
+          const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
+          const long long t0 = global_ns();
+          while (!mbar_try(bar, (idx / kNumBuf) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ================= MMA issuer (one lane) =================
+    if (lane == 0 && n_tiles > 0) {
+      mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
+      tc_fence_after();
+      auto issue_qk = [&](int t, int j) {
+        const int idx = 2 * j;
+        const uint32_t kbuf = smem_base + kOffKV + (idx % kNumBuf) * kTileBytes;
+        const uint32_t qbuf = smem_base + kOffQ + t * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
+          mma_ss(tmem + t * 128, make_desc(qbuf + off, 16, 1024), make_desc(kbuf + off, 16, 1024), kIdescQK, ks > 0);
+        }
+        mma_commit(smem_u32(&bars.s_full[t]));
+      };
+      auto issue_pv = [&](int t, int j) {
+        const int idx = 2 * j + 1;
+        const uint32_t vbuf = smem_base + kOffKV + (idx % kNumBuf) * kTileBytes;
+        const uint32_t pbuf = smem_base + kOffP + t * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kTileKeys / 16; ++ks) {
+          const uint32_t aoff = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
+          mma_ss(tmem + 256 + t * 128, make_desc(pbuf + aoff, 16, 1024), make_desc(vbuf + ks * 2048, kSlabBytes, 1024),
+                 kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        mma_commit(smem_u32(&bars.p_free[t]));
+      };
+      // tile 0 of both halves
+      mbar_wait(smem_u32(&bars.kv_full[0]), 0, abort_flag, P.status);
+      tc_fence_after();
+      for (int t = 0; t < 2; ++t) if (t_tiles[t] > 0) issue_qk(t, 0);
+      mma_commit(smem_u32(&bars.kv_empty[0]));
+      for (int j = 0; j < n_tiles; ++j) {
+        if (j + 1 < n_tiles) {
+          const int idx = 2 * (j + 1);
+          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+          for (int t = 0; t < 2; ++t) {
+            if (j + 1 < t_tiles[t]) {
+              mbar_wait(smem_u32(&bars.s_free[t]), j & 1, abort_flag, P.status);   // S_t(j) is in registers
+              tc_fence_after();
+              issue_qk(t, j + 1);
+            }
+          }
+          mma_commit(smem_u32(&bars.kv_empty[idx % kNumBuf]));
+        }
+        {
+          const int idx = 2 * j + 1;
+          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+          if (kv_end < kv_begin + (j + 1) * kTileKeys) {
+            // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
+            // them so that weight 0 times leftover bits cannot produce NaN
+            const int first = kv_end - (kv_begin + j * kTileKeys);
+            uint8_t* vgen = smem_gen + kOffKV + (idx % kNumBuf) * kTileBytes;
+            for (int rr = first; rr < kTileKeys; ++rr)
+              for (int c = 0; c < 16; ++c)
+                *reinterpret_cast<uint4*>(vgen + (c >> 3) * kSlabBytes + rr * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+            fence_async_smem();
+          }
+          for (int t = 0; t < 2; ++t) {
+            if (j < t_tiles[t]) {
+              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
+              tc_fence_after();
+              issue_pv(t, j);
+            }
+          }
+          mma_commit(smem_u32(&bars.kv_empty[idx % kNumBuf]));
+        }
+      }
+      // every MMA has completed (commits arrive in issue order) before this thread leaves
+      {
+        const int idx = 2 * n_tiles - 1;
+        mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+      }
+    }
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    // ================= softmax warpgroups =================
+    const int t = warp >> 2;                                   // 0 = A, 1 = B
+    const int row = ((warp & 3) << 5) | lane;                  // row of the 128-row tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
+    const int r = item_row0 + t * 128 + row;
+    const bool valid = r < R;
+    const int qi = r / g.G, hd = kvh * g.G + (r - qi * g.G);
+    const int my_tiles = t_tiles[t];
+    const int limit = valid ? min(t_end[t], seg.p + qi + 1) : t_end[t];   // keys j < limit are visible
+
+    // ---- stage this row of Q (or zeros) as an MMA operand ----
+    {
+      uint8_t* qrow = smem_gen + kOffQ + t * kTileBytes + row * 128;
+      const uint4* src = reinterpret_cast<const uint4*>(P.q + ((long long)(seg.q_off + qi) * g.Hq + hd) * D);
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(qrow + (c >> 3) * kSlabBytes + (((c & 7) ^ (row & 7)) << 4)) = v;
+      }
+      fence_async_smem();
+      mbar_arrive(smem_u32(&bars.q_full));
+    }
+
+    float m = -INFINITY, l = 0.f;       // running max (base-2, scaled) and sum
+    const float sl2 = P.scale_log2e;
+    const uint32_t s_addr = tmem + lane_addr + t * 128;
+    const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
+    uint8_t* prow = smem_gen + kOffP + t * kTileBytes + row * 128;
+
+    for (int j = 0; j < my_tiles; ++j) {
+      mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
+      tc_fence_after();
+      float s[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bars.s_free[t]));
+      const int tile_key0 = kv_begin + j * kTileKeys;
+      if (tile_key0 + kTileKeys > t_min_limit[t]) {            // uniform over the warpgroup
+        const int vis = limit - tile_key0;
+#pragma unroll
+        for (int c = 0; c < 128; ++c) if (c >= vis) s[c] = -INFINITY;
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, s[c]);
+      mx *= sl2;                                               // scale > 0 on this path
+      float m_new = m;
+      if (mx > m + kRescaleThreshold || m == -INFINITY) m_new = fmaxf(m, mx);
+      const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);   // m = -inf -> 0
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        mbar_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, abort_flag, P.status);   // O_t holds tiles < j
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(o_addr + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] *= alpha;
+          tmem_st32(o_addr + c * 32, o);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+      }
+      m = m_new;
+      const float mu = (m == -INFINITY) ? 0.f : m;
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 128; ++c) { s[c] = fast_exp2(fmaf(s[c], sl2, -mu)); sum += s[c]; }
+      l = l * alpha + sum;
+      if (j > 0) mbar_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, abort_flag, P.status);   // P buffer is free
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        uint4 v;
+        v.x = pack_bf16(s[c * 8 + 0], s[c * 8 + 1]);
+        v.y = pack_bf16(s[c * 8 + 2], s[c * 8 + 3]);
+        v.z = pack_bf16(s[c * 8 + 4], s[c * 8 + 5]);
+        v.w = pack_bf16(s[c * 8 + 6], s[c * 8 + 7]);
+        *reinterpret_cast<uint4*>(prow + (c >> 3) * kSlabBytes + (((c & 7) ^ (row & 7)) << 4)) = v;
+      }
+      fence_async_smem();
+      mbar_arrive(smem_u32(&bars.p_full[t]));
+    }
+
+    // ---- epilogue: O / l and LSE ----
+    const float kLn2 = 0.6931471805599453f;
+    if (my_tiles > 0) {
+      mbar_wait(smem_u32(&bars.p_free[t]), (my_tiles - 1) & 1, abort_flag, P.status);
+      tc_fence_after();
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const float e2 = l > 0.f ? m + log2f(l) : -INFINITY;
+    const long long orow = (long long)(seg.q_off + qi) * g.Hq + hd;
+    const long long prow_idx = seg.part_base + (long long)(split * seg.n + qi) * g.Hq + hd;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float o[32];
+      if (my_tiles > 0) {                 // uniform over the warpgroup
+        tmem_ld32(o_addr + c * 32, o);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = 0.f;
+      }
+      if (valid) {
+        if (direct) {
+          uint4* dst = reinterpret_cast<uint4*>(P.out + orow * D + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 v;
+            v.x = pack_bf16(o[i * 8 + 0] * inv, o[i * 8 + 1] * inv);
+            v.y = pack_bf16(o[i * 8 + 2] * inv, o[i * 8 + 3] * inv);
+            v.z = pack_bf16(o[i * 8 + 4] * inv, o[i * 8 + 5] * inv);
+            v.w = pack_bf16(o[i * 8 + 6] * inv, o[i * 8 + 7] * inv);
+            dst[i] = v;
+          }
+        } else {
+          float4* dst = reinterpret_cast<float4*>(P.part_o + prow_idx * D + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[i * 4] * inv, o[i * 4 + 1] * inv, o[i * 4 + 2] * inv, o[i * 4 + 3] * inv);
+        }
+      }
+    }
+    if (valid) {
+      if (direct) { if (P.lse != nullptr) P.lse[orow] = e2 * kLn2; }
+      else P.part_lse[prow_idx] = e2;
+    }
+    tc_fence_before();
+  }
+
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace umma
+
+cudaError_t attend_umma_init() {
+  return cudaFuncSetAttribute(umma::attend_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
+}
+
+cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s) {
+  if (p.n_items <= 0) return cudaSuccess;
+  umma::attend_umma_kernel<<<p.n_items, umma::kThreads, umma::kSmemBytes, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace tide

@@ -7,6 +7,7 @@
 // back last-to-first.  Every call validates completely before it changes anything.
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -72,6 +73,7 @@ struct tide_kv {
   cudaEvent_t ev_append[2] = {nullptr, nullptr};
   cudaEvent_t ev_attend[4] = {nullptr, nullptr, nullptr, nullptr};
   bool have_append_times = false, have_attend_times = false;
+  int umma_min_rows = kUmmaTileRows;  // packed rows from which a resume row takes the tcgen05 path
 };
 
 namespace {
@@ -209,7 +211,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->d_part_o = (float*)(kv->ws + lay.off_part_o);
   kv->d_part_lse = (float*)(kv->ws + lay.off_part_lse);
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
-  ok = ok && attend_kernels_init() == cudaSuccess;
+  ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
   for (int i = 0; ok && i < kSlots; ++i) {
@@ -225,6 +227,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->len.assign((size_t)cfg->max_tasks, 0);
   kv->pages.resize((size_t)cfg->max_tasks);
   kv->mark.assign((size_t)cfg->max_tasks, 0);
+  if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
   *out = kv;
   return TIDE_OK;
@@ -468,7 +471,9 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   if (total_q > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
 
   // ---- plan: one segment per row, decode-style (<= 16 packed rows) or tile-style ----
-  struct RowPlan { int b; bool decode; int n_mtiles; long long items; };
+  enum { kDec = 0, kTile = 1, kUmma = 2 };
+  struct RowPlan { int b; int kind; int n_mtiles; long long items; };
+  const bool umma_ok = g.D == 128 && scale > 0.f;
   std::vector<RowPlan> plan((size_t)n_rows);
   long long w_dec = 0, w_tile = 0, items_tile_nosplit = 0;
   {
@@ -477,10 +482,10 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
       const int R = r.q_len * g.G;
       RowPlan& p = plan[(size_t)b];
       p.b = b;
-      p.decode = R <= kDecodeTileRows;
-      p.n_mtiles = p.decode ? 1 : ceil_div(R, kMmaTileRows);
+      p.kind = R <= kDecodeTileRows ? kDec : (umma_ok && R >= kv->umma_min_rows ? kUmma : kTile);
+      p.n_mtiles = p.kind == kDec ? 1 : ceil_div(R, p.kind == kUmma ? 2 * kUmmaTileRows : kMmaTileRows);
       p.items = (long long)g.Hkv * p.n_mtiles;
-      if (p.decode) w_dec += (long long)g.Hkv * r.ctx_len;
+      if (p.kind == kDec) w_dec += (long long)g.Hkv * r.ctx_len;
       else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
     }
   }
@@ -489,19 +494,19 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   long long chunk_tile = (items_tile_nosplit >= target / 2)
                              ? (1LL << 30)
                              : std::max<long long>(2048, align_up((size_t)(w_tile / target + 1), kStageKeys));
-  std::vector<Segment> seg_dec, seg_tile, seg_merge;
-  long long items_dec = 0, items_tile = 0, part_rows = 0, merge_rows = 0;
+  std::vector<Segment> seg_dec, seg_tile, seg_umma, seg_merge;
+  long long items_dec = 0, items_tile = 0, items_umma = 0, part_rows = 0, merge_rows = 0;
   for (int attempt = 0; attempt < 40; ++attempt) {
-    seg_dec.clear(); seg_tile.clear();
+    seg_dec.clear(); seg_tile.clear(); seg_umma.clear();
     part_rows = 0;
     long long qoff = 0;
     for (int b = 0; b < n_rows; ++b) {
       const tide_row_t& r = rows[b];
       const RowPlan& p = plan[(size_t)b];
-      const long long chunk_target = p.decode ? chunk_dec : chunk_tile;
+      const long long chunk_target = p.kind == kDec ? chunk_dec : chunk_tile;
       int n_splits = (int)std::min<long long>(kMaxSplits, ((long long)r.ctx_len + chunk_target - 1) / chunk_target);
       n_splits = std::max(1, n_splits);
-      int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), kStageKeys);
+      int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), 2 * kStageKeys);
       n_splits = ceil_div(r.ctx_len, chunk);
       Segment s{};
       s.table_off = r.task * g.max_pages_per_task;
@@ -513,7 +518,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
       s.chunk = chunk;
       s.part_base = 0;
       if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
-      (p.decode ? seg_dec : seg_tile).push_back(s);
+      (p.kind == kDec ? seg_dec : p.kind == kTile ? seg_tile : seg_umma).push_back(s);
       qoff += r.q_len;
     }
     if (part_rows <= kv->lay.part_rows) break;
@@ -527,8 +532,9 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   };
   std::stable_sort(seg_dec.begin(), seg_dec.end(), heavier);
   std::stable_sort(seg_tile.begin(), seg_tile.end(), heavier);
+  std::stable_sort(seg_umma.begin(), seg_umma.end(), heavier);
   long long part_cursor = 0;
-  for (auto* v : {&seg_dec, &seg_tile}) {
+  for (auto* v : {&seg_dec, &seg_tile, &seg_umma}) {
     long long base = 0;
     for (Segment& s : *v) {
       s.item_base = (int32_t)base;
@@ -542,9 +548,9 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
         seg_merge.push_back(s);
       }
     }
-    (v == &seg_dec ? items_dec : items_tile) = base;
+    (v == &seg_dec ? items_dec : v == &seg_tile ? items_tile : items_umma) = base;
   }
-  const size_t n_all = seg_dec.size() + seg_tile.size() + seg_merge.size();
+  const size_t n_all = seg_dec.size() + seg_tile.size() + seg_umma.size() + seg_merge.size();
   if (n_all * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
 
   cudaStream_t st = (cudaStream_t)stream;
@@ -554,7 +560,8 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   Segment* h = (Segment*)(slot->host + 256);
   std::copy(seg_dec.begin(), seg_dec.end(), h);
   std::copy(seg_tile.begin(), seg_tile.end(), h + seg_dec.size());
-  std::copy(seg_merge.begin(), seg_merge.end(), h + seg_dec.size() + seg_tile.size());
+  std::copy(seg_umma.begin(), seg_umma.end(), h + seg_dec.size() + seg_tile.size());
+  std::copy(seg_merge.begin(), seg_merge.end(), h + seg_dec.size() + seg_tile.size() + seg_umma.size());
   if (cudaMemcpyAsync(slot->dev + 256, h, n_all * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
   const Segment* d = (const Segment*)(slot->dev + 256);
 
@@ -582,10 +589,15 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
     if (launch_attend_tile(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
+  if (items_umma > 0) {
+    ap.segs = d + seg_dec.size() + seg_tile.size(); ap.n_segs = (int)seg_umma.size(); ap.n_items = (int)items_umma;
+    if (launch_attend_umma(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++launches;
+  }
   if (kv->profiling) cudaEventRecord(kv->ev_attend[2], st);
   if (merge_rows > 0) {
     MergeParams mp;
-    mp.segs = d + seg_dec.size() + seg_tile.size();
+    mp.segs = d + seg_dec.size() + seg_tile.size() + seg_umma.size();
     mp.n_segs = (int)seg_merge.size();
     mp.n_rows = (int)merge_rows;
     mp.part_o = kv->d_part_o; mp.part_lse = kv->d_part_lse;
@@ -599,7 +611,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   }
   if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   kv->last_decode_items = items_dec;
-  kv->last_prefill_items = items_tile;
+  kv->last_prefill_items = items_tile + items_umma;
   kv->last_merge_rows = merge_rows;
   kv->last_launches = launches + kv->append_launches;
   kv->append_launches = 0;

@@ -99,7 +99,9 @@ cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int len, 
 cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s);
 cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);
+cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s);
 cudaError_t attend_kernels_init();
+cudaError_t attend_umma_init();
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------------------
