@@ -132,7 +132,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
 
-    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank)
+    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank, n_tasks=args.tasks, len_div=args.len_div)
     kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank)
     rows = tide.rows_array(w.rows())
     ids = np.asarray(w.task, dtype=np.int32)
@@ -153,6 +153,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
         rollback()
@@ -161,9 +163,8 @@ def run_ours(args):
     plan = kv.last_plan()
 
     # ---- timed region 1: K whole steps, device time ----
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier()
+    sampler.lines.clear()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
@@ -218,6 +219,7 @@ def run_ours(args):
     tflops = res_flops_all / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0
 
     if rank == 0:
+        reduced = args.tasks is not None or args.len_div != 1
         n_app = int(w.n_new.sum())
         app_bytes = 2 * w.kv_bytes_per_token() * n_app
         use_tensor = res_flops > 0 and tile_ms >= dec_ms
@@ -239,7 +241,8 @@ def run_ours(args):
             "append_prefill_tflops": tflops,
             "phase_ms": {"append": app_ms, "decode_kernel": dec_ms, "tile_kernel": tile_ms, "merge": mrg_ms},
             "append_gbs": app_bytes / (ph_ms["append"] * 1e-3) / 1e9 if ph_ms["append"] > 0 else 0.0,
-            "config": {"workload": f"configs[{args.config - 1}]: {w.name}", "tasks": w.B,
+            "config": {"workload": f"configs[{args.config - 1}]: {w.name}" + (" (REDUCED for a profiler capture)" if reduced else ""),
+                       "tasks": w.B,
                        "decode_rows": int((w.n_new == 1).sum()), "resume_rows": int((w.n_new > 1).sum()),
                        "new_tokens": n_app, "prefix_tokens": int(w.prefix.sum()),
                        "heads": f"{w.Hq}q/{w.Hkv}kv", "head_dim": w.D, "page_size": w.S,
@@ -342,6 +345,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=3, help="BASELINE.json configs[config-1]; default the mixed resume batch")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tasks", type=int, default=None, help="fewer tasks (profiler captures only)")
+    ap.add_argument("--len-div", type=int, default=1, help="divide every length bound (profiler captures only)")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
     if args.impl == "reference":

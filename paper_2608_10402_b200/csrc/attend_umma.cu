@@ -13,12 +13,14 @@
 // and V tiles of 128 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
 // 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.
 //   S_t = Q_t . K_j^T   (SS MMA, 128x128x128, fp32 in TMEM)       t in {A, B}
-//   softmax WG t: TMEM -> registers, max / exp2 / sum, P_t as bf16 into shared memory
-//   O_t += P_t . V_j    (SS MMA, V tile used MN-major)
-// QK of tile j+1 is issued as soon as the softmax warpgroup has pulled S_t(j) into registers, so the tensor
-// pipe works on the other tile / the next keys while exponentials are computed.  O is only rescaled when a
-// row's running maximum grows by more than 2^8 (the final normalisation uses the same stale maximum, so the
-// result is exact); that happens on the first tiles only.
+//   softmax WG t: TMEM -> registers, max / exp2 / sum, P_t as packed bf16 back into the first 64 columns of
+//                 S_t (TMEM), so no shared memory and no proxy fence is spent on P
+//   O_t += P_t . V_j    (TS MMA: A operand from TMEM, V tile used MN-major)
+// The two halves ping-pong: while warpgroup A computes exponentials the tensor pipe runs PV_B(j) and
+// QK_B(j+1), and vice versa.  Shared memory holds only Q (64 KB) and a 5-deep ring of K / V tiles, so loads
+// run more than two key tiles ahead of the MMAs.  O is only rescaled when a row's running maximum grows by
+// more than 2^8 (the final normalisation uses the same stale maximum, so the result is exact); that happens
+// on the first tiles only.
 // Every wait is bounded; a wait that runs out sets TIDE_ERR_DEVICE_TIMEOUT and the CTA drains and exits.
 #include <climits>
 
@@ -31,13 +33,12 @@ namespace umma {
 constexpr int D = 128;
 constexpr int kTileKeys = 128;
 constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA issuer, 2 idle warps}
-constexpr int kNumBuf = 3;                          // ring of K / V tiles: K0 V0 K1 V1 ...
+constexpr int kNumBuf = 5;                          // ring of K / V tiles: K0 V0 K1 V1 ...
 constexpr int kTileBytes = 128 * 128 * 2;           // one operand tile (Q half, P, K or V): 32 KB
 constexpr int kSlabBytes = 128 * 128;               // 128 rows x 128 bytes
 constexpr int kOffQ = 0;                            // Q_A, Q_B
-constexpr int kOffP = 2 * kTileBytes;               // P_A, P_B
-constexpr int kOffKV = 4 * kTileBytes;
-constexpr int kSmemBytes = (4 + kNumBuf) * kTileBytes + 1024;
+constexpr int kOffKV = 2 * kTileBytes;
+constexpr int kSmemBytes = (2 + kNumBuf) * kTileBytes + 1024;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
 
 // instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
@@ -59,6 +60,15 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, 
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// A operand (16-bit, two K-elements per 32-bit column, one row per lane) read from TMEM
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -99,6 +109,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         "r"(__float_as_uint(v[31]))
       : "memory");
 }
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -106,10 +127,9 @@ struct Bars {
   uint64_t kv_full[kNumBuf];
   uint64_t kv_empty[kNumBuf];
   uint64_t q_full;
-  uint64_t s_full[2];
-  uint64_t s_free[2];
-  uint64_t p_full[2];
-  uint64_t p_free[2];
+  uint64_t s_full[2];   // S_t(j) is in TMEM (and every earlier MMA, PV_t(j-1) included, has retired)
+  uint64_t p_full[2];   // P_t(j) is in TMEM
+  uint64_t o_full[2];   // the last PV_t has retired
 };
 
 __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendParams P) {
@@ -159,9 +179,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     mbar_init(smem_u32(&bars.q_full), 256);
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.s_free[t]), 128);
       mbar_init(smem_u32(&bars.p_full[t]), 128);
-      mbar_init(smem_u32(&bars.p_free[t]), 1);
+      mbar_init(smem_u32(&bars.o_full[t]), 1);
     }
     mbar_fence_init();
   }
@@ -230,55 +249,44 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       auto issue_pv = [&](int t, int j) {
         const int idx = 2 * j + 1;
         const uint32_t vbuf = smem_base + kOffKV + (idx % kNumBuf) * kTileBytes;
-        const uint32_t pbuf = smem_base + kOffP + t * kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < kTileKeys / 16; ++ks) {
-          const uint32_t aoff = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
-          mma_ss(tmem + 256 + t * 128, make_desc(pbuf + aoff, 16, 1024), make_desc(vbuf + ks * 2048, kSlabBytes, 1024),
-                 kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-        }
-        mma_commit(smem_u32(&bars.p_free[t]));
+        for (int ks = 0; ks < kTileKeys / 16; ++ks)
+          mma_ts(tmem + 256 + t * 128, tmem + t * 128 + ks * 8, make_desc(vbuf + ks * 2048, kSlabBytes, 1024), kIdescPV,
+                 (j > 0 || ks > 0) ? 1u : 0u);
       };
-      // tile 0 of both halves
-      mbar_wait(smem_u32(&bars.kv_full[0]), 0, abort_flag, P.status);
+      auto wait_full = [&](int idx) {
+        mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+      };
+      wait_full(0);
       tc_fence_after();
       for (int t = 0; t < 2; ++t) if (t_tiles[t] > 0) issue_qk(t, 0);
       mma_commit(smem_u32(&bars.kv_empty[0]));
       for (int j = 0; j < n_tiles; ++j) {
-        if (j + 1 < n_tiles) {
-          const int idx = 2 * (j + 1);
-          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
-          for (int t = 0; t < 2; ++t) {
-            if (j + 1 < t_tiles[t]) {
-              mbar_wait(smem_u32(&bars.s_free[t]), j & 1, abort_flag, P.status);   // S_t(j) is in registers
-              tc_fence_after();
-              issue_qk(t, j + 1);
-            }
-          }
-          mma_commit(smem_u32(&bars.kv_empty[idx % kNumBuf]));
+        const int vidx = 2 * j + 1;
+        wait_full(vidx);
+        if (kv_end < kv_begin + (j + 1) * kTileKeys) {
+          // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
+          // them so that weight 0 times leftover bits cannot produce NaN
+          const int first = kv_end - (kv_begin + j * kTileKeys);
+          uint8_t* vgen = smem_gen + kOffKV + (vidx % kNumBuf) * kTileBytes;
+          for (int rr = first; rr < kTileKeys; ++rr)
+            for (int c = 0; c < 16; ++c)
+              *reinterpret_cast<uint4*>(vgen + (c >> 3) * kSlabBytes + rr * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+          fence_async_smem();
         }
-        {
-          const int idx = 2 * j + 1;
-          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
-          if (kv_end < kv_begin + (j + 1) * kTileKeys) {
-            // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
-            // them so that weight 0 times leftover bits cannot produce NaN
-            const int first = kv_end - (kv_begin + j * kTileKeys);
-            uint8_t* vgen = smem_gen + kOffKV + (idx % kNumBuf) * kTileBytes;
-            for (int rr = first; rr < kTileKeys; ++rr)
-              for (int c = 0; c < 16; ++c)
-                *reinterpret_cast<uint4*>(vgen + (c >> 3) * kSlabBytes + rr * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
-            fence_async_smem();
+        const bool more = j + 1 < n_tiles;
+        if (more) wait_full(vidx + 1);
+        for (int t = 0; t < 2; ++t) {
+          if (j < t_tiles[t]) {
+            mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
+            tc_fence_after();
+            issue_pv(t, j);
+            if (j + 1 < t_tiles[t]) issue_qk(t, j + 1);             // overwrites S_t / P_t after PV_t(j), in order
+            else mma_commit(smem_u32(&bars.o_full[t]));
           }
-          for (int t = 0; t < 2; ++t) {
-            if (j < t_tiles[t]) {
-              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
-              tc_fence_after();
-              issue_pv(t, j);
-            }
-          }
-          mma_commit(smem_u32(&bars.kv_empty[idx % kNumBuf]));
         }
+        mma_commit(smem_u32(&bars.kv_empty[vidx % kNumBuf]));
+        if (more) mma_commit(smem_u32(&bars.kv_empty[(vidx + 1) % kNumBuf]));
       }
       // every MMA has completed (commits arrive in issue order) before this thread leaves
       {
@@ -316,7 +324,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const float sl2 = P.scale_log2e;
     const uint32_t s_addr = tmem + lane_addr + t * 128;
     const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
-    uint8_t* prow = smem_gen + kOffP + t * kTileBytes + row * 128;
 
     for (int j = 0; j < my_tiles; ++j) {
       mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
@@ -325,24 +332,28 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
       tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&bars.s_free[t]));
       const int tile_key0 = kv_begin + j * kTileKeys;
       if (tile_key0 + kTileKeys > t_min_limit[t]) {            // uniform over the warpgroup
         const int vis = limit - tile_key0;
 #pragma unroll
         for (int c = 0; c < 128; ++c) if (c >= vis) s[c] = -INFINITY;
       }
-      float mx = -INFINITY;
+      // independent partial reductions: a single 128-long dependent chain would expose its latency
+      float mxp[8];
 #pragma unroll
-      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, s[c]);
+      for (int k = 0; k < 8; ++k) mxp[k] = fmaxf(s[k], s[k + 8]);
+#pragma unroll
+      for (int c = 16; c < 128; c += 16) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mxp[k] = fmaxf(mxp[k], fmaxf(s[c + k], s[c + k + 8]));
+      }
+      float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
       mx *= sl2;                                               // scale > 0 on this path
       float m_new = m;
       if (mx > m + kRescaleThreshold || m == -INFINITY) m_new = fmaxf(m, mx);
       const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);   // m = -inf -> 0
       if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-        mbar_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, abort_flag, P.status);   // O_t holds tiles < j
-        tc_fence_after();
+        // O_t holds tiles < j: S_t(j) was committed after PV_t(j-1)
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           float o[32];
@@ -352,33 +363,36 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           for (int i = 0; i < 32; ++i) o[i] *= alpha;
           tmem_st32(o_addr + c * 32, o);
         }
-        tmem_wait_st();
-        tc_fence_before();
       }
       m = m_new;
       const float mu = (m == -INFINITY) ? 0.f : m;
-      float sum = 0.f;
+      float sp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 128; ++c) { s[c] = fast_exp2(fmaf(s[c], sl2, -mu)); sum += s[c]; }
-      l = l * alpha + sum;
-      if (j > 0) mbar_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, abort_flag, P.status);   // P buffer is free
+      for (int h = 0; h < 2; ++h) {
+        uint32_t pk[32];
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        uint4 v;
-        v.x = pack_bf16(s[c * 8 + 0], s[c * 8 + 1]);
-        v.y = pack_bf16(s[c * 8 + 2], s[c * 8 + 3]);
-        v.z = pack_bf16(s[c * 8 + 4], s[c * 8 + 5]);
-        v.w = pack_bf16(s[c * 8 + 6], s[c * 8 + 7]);
-        *reinterpret_cast<uint4*>(prow + (c >> 3) * kSlabBytes + (((c & 7) ^ (row & 7)) << 4)) = v;
+        for (int c = 0; c < 64; c += 8) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float e = fast_exp2(fmaf(s[h * 64 + c + k], sl2, -mu));
+            s[h * 64 + c + k] = e;
+            sp[k] += e;
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) pk[(c >> 1) + k] = pack_bf16(s[h * 64 + c + 2 * k], s[h * 64 + c + 2 * k + 1]);
+        }
+        tmem_st32u(s_addr + h * 32, pk);                       // P_t over the first 64 columns of S_t
       }
-      fence_async_smem();
+      l = l * alpha + (((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7])));
+      tmem_wait_st();
+      tc_fence_before();
       mbar_arrive(smem_u32(&bars.p_full[t]));
     }
 
     // ---- epilogue: O / l and LSE ----
     const float kLn2 = 0.6931471805599453f;
     if (my_tiles > 0) {
-      mbar_wait(smem_u32(&bars.p_free[t]), (my_tiles - 1) & 1, abort_flag, P.status);
+      mbar_wait(smem_u32(&bars.o_full[t]), 0, abort_flag, P.status);
       tc_fence_after();
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
