@@ -162,6 +162,26 @@ int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items,
 int tide_set_profiling(tide_kv_t* kv, int enable);
 int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile_ms, float* merge_ms);
 
+/* (The paper has no counterpart to this call; it exists for callers of this library.)
+ * Attention for decode-style rows (q_len * Hq/Hkv <= 16) that allocates nothing, neither on the device nor on
+ * the host.  tide_attend parks the partial results of its KV splits and its row descriptors in the workspace
+ * that the caller allocated; this variant keeps both in a fixed array compiled into the library (about 8 MB of
+ * device memory on every GPU that loads the library, held until the process exits).  It is meant for callers
+ * that cannot allocate at the time they need attention: code running while a CUDA graph is being captured in
+ * global mode, where cudaMalloc is refused; processes whose framework allocator already owns the whole device,
+ * so a fresh cudaMalloc fails; and steps that cannot afford the device-wide synchronisation cudaMalloc implies.
+ * Same semantics, arguments and results as tide_attend restricted to such rows, with the library's own page
+ * table.  Limits: at most TIDE_STATIC_MAX_ROWS rows per call (more returns TIDE_ERR_WORKSPACE), decode-style
+ * rows only (others return TIDE_ERR_INVALID_ARG); long rows are split over KV only as far as the fixed array
+ * allows.  The first call on a device looks up the array's device address; make that call before any stream
+ * capture begins.  Every call uses the same array and overwrites what the previous call left there (nothing in
+ * it needs clearing between calls), so two calls whose kernels may overlap on the GPU (different streams) race:
+ * keep the calls of one process on one stream, or order them with events. */
+#define TIDE_STATIC_MAX_ROWS 64
+int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows /*host*/,
+                              const void* q /*device*/, float scale, void* out /*device*/,
+                              float* lse /*device or NULL*/, void* stream);
+
 const char* tide_strerror(int code);
 
 #ifdef __cplusplus

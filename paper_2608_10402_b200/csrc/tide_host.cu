@@ -703,6 +703,20 @@ int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile
   return TIDE_OK;
 }
 
+// Read-only view of a handle for attend_static.cu (not part of the public header).
+int tide_internal_view(tide_kv_t* kv, Geom* g, const uint8_t** pool, const int32_t** table, int** status,
+                       const int32_t** len, const uint8_t** live, int32_t* max_tasks) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  *g = kv->g;
+  *pool = kv->pool;
+  *table = kv->d_table;
+  *status = kv->d_status;
+  *len = kv->len.data();
+  *live = kv->live.data();
+  *max_tasks = kv->cfg.max_tasks;
+  return TIDE_OK;
+}
+
 int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,
                    int64_t* kernel_launches) {
   if (kv == nullptr) return TIDE_ERR_INVALID_ARG;

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libtide.so")
 OK = 0
 ERR_INVALID_ARG, ERR_UNKNOWN_TASK, ERR_TASK_EXISTS, ERR_DUPLICATE_TASK = -1, -2, -3, -4
 ERR_NO_PAGES, ERR_TABLE_FULL, ERR_CTX_RANGE, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = -5, -6, -7, -8, -9, -10
+STATIC_MAX_ROWS = 64
 
 
 class TideError(RuntimeError):
@@ -45,7 +46,7 @@ EXPORTS = [
     "tide_strerror", "tide_kv_required_bytes", "tide_kv_create", "tide_kv_destroy", "tide_kv_reset",
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
-    "tide_set_profiling", "tide_phase_ms",
+    "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -170,6 +171,12 @@ class TideKV:
         arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
         _check(lib.tide_attend(self.handle, ctypes.c_int32(0), ctypes.c_int32(len(arr)), arr, _ptr(page_table), _ptr(q),
                                ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)), "tide_attend")
+
+    def attend_decode_static(self, rows, q, scale, out, lse=None, stream=None):
+        """tide_attend_decode_static: decode-style rows only, scratch in the library's fixed device array."""
+        arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
+        _check(lib.tide_attend_decode_static(self.handle, ctypes.c_int32(len(arr)), arr, _ptr(q), ctypes.c_float(scale),
+                                             _ptr(out), _ptr(lse), _stream(stream)), "tide_attend_decode_static")
 
     def step_host(self, rows, new_k, new_v, q, scale, out, lse=None, stream=None):
         arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
