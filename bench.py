@@ -132,7 +132,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
 
-    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank, n_tasks=args.tasks, len_div=args.len_div)
+    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank, n_tasks=args.tasks, len_div=args.len_div,
+                              pool_factor=args.pool_factor)
     kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank)
     rows = tide.rows_array(w.rows())
     ids = np.asarray(w.task, dtype=np.int32)
@@ -219,7 +220,7 @@ def run_ours(args):
     tflops = res_flops_all / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0
 
     if rank == 0:
-        reduced = args.tasks is not None or args.len_div != 1
+        reduced = args.tasks is not None or args.len_div != 1 or args.pool_factor is not None
         n_app = int(w.n_new.sum())
         app_bytes = 2 * w.kv_bytes_per_token() * n_app
         use_tensor = res_flops > 0 and tile_ms >= dec_ms
@@ -347,6 +348,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tasks", type=int, default=None, help="fewer tasks (profiler captures only)")
     ap.add_argument("--len-div", type=int, default=1, help="divide every length bound (profiler captures only)")
+    ap.add_argument("--pool-factor", type=float, default=None, help="pool pages / live pages (profiler captures only)")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
     if args.impl == "reference":
