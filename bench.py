@@ -120,7 +120,7 @@ def build_state(w, torch, tide, seed):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2608_10402_b200 import inputs, tide
+    from paper_2608_10402_b200 import inputs, replicas, tide
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -132,7 +132,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
 
-    w = inputs.make_workload(args.config, seed=1000 + args.config + 7919 * rank, n_tasks=args.tasks, len_div=args.len_div,
+    w = inputs.make_workload(args.config, seed=replicas.rank_seed(1000 + args.config, rank), n_tasks=args.tasks, len_div=args.len_div,
                               pool_factor=args.pool_factor)
     kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank)
     rows = tide.rows_array(w.rows())
@@ -208,16 +208,11 @@ def run_ours(args):
     # ---- numbers ----
     dec_bytes = w.decode_kv_bytes()
     res_flops = w.resume_flops()
-    t = torch.tensor([step_ms, ph_ms["decode"], ph_ms["tile"], ph_ms["append"], ph_ms["merge"], e2e_ms],
-                     device="cuda", dtype=torch.float64)
-    tot = torch.tensor([dec_bytes, res_flops], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-    step_ms, dec_ms, tile_ms, app_ms, mrg_ms, e2e_ms = [float(x) for x in t.tolist()]
-    dec_bytes_all, res_flops_all = [float(x) for x in tot.tolist()]
-    kv_gbs = dec_bytes_all / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
-    tflops = res_flops_all / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0
+    (step_ms, dec_ms, tile_ms, app_ms, mrg_ms, e2e_ms), (dec_bytes_all, res_flops_all) = replicas.reduce_step_stats(
+        [step_ms, ph_ms["decode"], ph_ms["tile"], ph_ms["append"], ph_ms["merge"], e2e_ms], [dec_bytes, res_flops],
+        world, dist, "cuda")
+    kv_gbs = replicas.whole_job_rate(dec_bytes_all, dec_ms) / 1e9
+    tflops = replicas.whole_job_rate(res_flops_all, tile_ms) / 1e12
 
     if rank == 0:
         reduced = args.tasks is not None or args.len_div != 1 or args.pool_factor is not None
