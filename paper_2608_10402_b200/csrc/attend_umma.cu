@@ -123,6 +123,26 @@ __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[3
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Optional cycle accounting (compile with -DTIDE_UMMA_TIMING): where the softmax warps and the MMA lane
+// spend their time, accumulated into 64-bit counters behind the status word.
+#ifdef TIDE_UMMA_TIMING
+#define TT_DECL long long tt_wait = 0, tt_wait2 = 0, tt_t0 = clock64(), tt_a
+#define TT_BEGIN tt_a = clock64()
+#define TT_END(acc) acc += clock64() - tt_a
+#define TT_FLUSH(i0, i1, i2)                                                                       \
+  do {                                                                                              \
+    unsigned long long* c = reinterpret_cast<unsigned long long*>(P.status) + 8;                   \
+    atomicAdd(c + (i0), (unsigned long long)tt_wait);                                               \
+    atomicAdd(c + (i1), (unsigned long long)tt_wait2);                                              \
+    atomicAdd(c + (i2), (unsigned long long)(clock64() - tt_t0));                                   \
+  } while (0)
+#else
+#define TT_DECL
+#define TT_BEGIN
+#define TT_END(acc)
+#define TT_FLUSH(i0, i1, i2)
+#endif
+
 struct Bars {
   uint64_t kv_full[kNumBuf];
   uint64_t kv_empty[kNumBuf];
@@ -233,6 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   } else if (warp == 9) {
     // ================= MMA issuer (one lane) =================
     if (lane == 0 && n_tiles > 0) {
+      TT_DECL;
       mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
       tc_fence_after();
       auto issue_qk = [&](int t, int j) {
@@ -255,7 +276,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
                  (j > 0 || ks > 0) ? 1u : 0u);
       };
       auto wait_full = [&](int idx) {
+        TT_BEGIN;
         mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+        TT_END(tt_wait2);
       };
       wait_full(0);
       tc_fence_after();
@@ -278,7 +301,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
         if (more) wait_full(vidx + 1);
         for (int t = 0; t < 2; ++t) {
           if (j < t_tiles[t]) {
+            TT_BEGIN;
             mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
+            TT_END(tt_wait);
             tc_fence_after();
             issue_pv(t, j);
             if (j + 1 < t_tiles[t]) issue_qk(t, j + 1);             // overwrites S_t / P_t after PV_t(j), in order
@@ -293,6 +318,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
         const int idx = 2 * n_tiles - 1;
         mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
       }
+      TT_FLUSH(2, 3, 4);
     }
   }
   } else {
@@ -325,8 +351,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const uint32_t s_addr = tmem + lane_addr + t * 128;
     const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
 
+    TT_DECL;
     for (int j = 0; j < my_tiles; ++j) {
+      TT_BEGIN;
       mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
+      TT_END(tt_wait);
       tc_fence_after();
       float s[128];
 #pragma unroll
@@ -392,9 +421,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     // ---- epilogue: O / l and LSE ----
     const float kLn2 = 0.6931471805599453f;
     if (my_tiles > 0) {
+      TT_BEGIN;
       mbar_wait(smem_u32(&bars.o_full[t]), 0, abort_flag, P.status);
+      TT_END(tt_wait2);
       tc_fence_after();
     }
+#ifdef TIDE_UMMA_TIMING
+    if (lane == 0 && (warp & 3) == 0) TT_FLUSH(0, 1, 5);
+#endif
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const float e2 = l > 0.f ? m + log2f(l) : -INFINITY;
     const long long orow = (long long)(seg.q_off + qi) * g.Hq + hd;

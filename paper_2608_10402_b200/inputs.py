@@ -218,3 +218,16 @@ def hashed_bf16_bits(task: int, start: int, count: int, Hkv: int, D: int, stream
     expo = (np.uint64(125) + ((x >> np.uint64(1)) & np.uint64(3))) << np.uint64(7)
     mant = (x >> np.uint64(3)) & np.uint64(0x7F)
     return (sign | expo | mant).astype(np.uint16)
+
+
+def hashed_bf16_bits_torch(torch, task: int, start: int, count: int, Hkv: int, D: int, stream: int, device="cuda"):
+    """The same filler as hashed_bf16_bits, produced on `device` with torch integer ops (int16 bit patterns)."""
+    pos = torch.arange(start, start + count, dtype=torch.int64, device=device)[:, None, None]
+    h = torch.arange(Hkv, dtype=torch.int64, device=device)[None, :, None]
+    d = torch.arange(D, dtype=torch.int64, device=device)[None, None, :]
+    x = (pos * 0x9E3779B1 + h * 0x85EBCA77 + d * 0xC2B2AE3D + int(task) * 0x27D4EB2F + int(stream) * 0x165667B1) & 0xFFFFFFFF
+    x = x ^ (x >> 15)
+    x = (x * 0x2C1B3C6D) & 0xFFFFFFFF
+    x = x ^ (x >> 12)
+    bits = ((x & 1) << 15) | ((125 + ((x >> 1) & 3)) << 7) | ((x >> 3) & 0x7F)
+    return bits.to(torch.int32).to(torch.int16)   # two's-complement wrap keeps the 16 bit pattern
