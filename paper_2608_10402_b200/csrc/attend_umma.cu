@@ -10,17 +10,18 @@
 // (packed row, key) pair against Hkv*D*4 bytes per key shared by all packed rows.
 //
 // CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warp 8 streams K
-// and V tiles of 128 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
-// 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.
-//   S_t = Q_t . K_j^T   (SS MMA, 128x128x128, fp32 in TMEM)       t in {A, B}
-//   softmax WG t: TMEM -> registers, max / exp2 / sum, P_t as packed bf16 back into the first 64 columns of
-//                 S_t (TMEM), so no shared memory and no proxy fence is spent on P
-//   O_t += P_t . V_j    (TS MMA: A operand from TMEM, V tile used MN-major)
-// The two halves ping-pong: while warpgroup A computes exponentials the tensor pipe runs PV_B(j) and
-// QK_B(j+1), and vice versa.  Shared memory holds only Q (64 KB) and a 5-deep ring of K / V tiles, so loads
-// run more than two key tiles ahead of the MMAs.  O is only rescaled when a row's running maximum grows by
-// more than 2^8 (the final normalisation uses the same stale maximum, so the result is exact); that happens
-// on the first tiles only.
+// and V tiles of 64 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
+// 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.  TMEM (512 columns):
+//   Q_A Q_B   2 x 64   the queries as packed bf16, staged once per item
+//   S_A S_B   2 x 64   fp32 logits of one 64-key tile; P (packed bf16) overwrites the first 32 columns
+//   O_A O_B   2 x 128  fp32 output accumulators
+//   S_t = Q_t . K_j^T   TS MMA, 128x64x16 x 8     O_t += P_t . V_j   TS MMA, 128x128x16 x 4 (V MN-major)
+// Both products take their A operand from TMEM: an MMA whose two operands both come from shared memory
+// (128x128x16, 8 KB per instruction) was measured at ~146 cycles against ~90 for the TMEM-A form, i.e. it is
+// bound by shared-memory operand fetch; with Q in TMEM shared memory only feeds K and V (64 B per cycle) and
+// is free for a deep K/V ring.  The two halves ping-pong: while warpgroup A computes exponentials the tensor
+// pipe runs PV_B(j) and QK_B(j+1), and vice versa.  O is only rescaled when a row's running maximum grows by
+// more than 2^8 (the final normalisation uses the same stale maximum, so the result is exact).
 // Every wait is bounded; a wait that runs out sets TIDE_ERR_DEVICE_TIMEOUT and the CTA drains and exits.
 #include <climits>
 
@@ -31,19 +32,20 @@ namespace tide {
 namespace umma {
 
 constexpr int D = 128;
-constexpr int kTileKeys = 128;
+constexpr int kTileKeys = 64;
 constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA issuer, 2 idle warps}
-constexpr int kNumBuf = 5;                          // ring of K / V tiles: K0 V0 K1 V1 ...
-constexpr int kTileBytes = 128 * 128 * 2;           // one operand tile (Q half, P, K or V): 32 KB
-constexpr int kSlabBytes = 128 * 128;               // 128 rows x 128 bytes
-constexpr int kOffQ = 0;                            // Q_A, Q_B
-constexpr int kOffKV = 2 * kTileBytes;
-constexpr int kSmemBytes = (2 + kNumBuf) * kTileBytes + 1024;
+constexpr int kNumBuf = 6;                          // ring of (K tile, V tile) slots
+constexpr int kTileBytes = kTileKeys * D * 2;       // one K or V tile: 16 KB
+constexpr int kSlotBytes = 2 * kTileBytes;          // K tile then V tile
+constexpr int kSlabBytes = kTileKeys * 128;         // 64 rows x 128 bytes
+constexpr int kSmemBytes = kNumBuf * kSlotBytes + 1024;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
+constexpr uint32_t kColQ = 0, kColS = 128, kColO = 256;
 
-// instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+// instruction descriptor: fp32 accumulate, bf16 A and B, M = 128; bit 16 = B is MN-major
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase | ((64u >> 3) << 17);                  // N = 64 keys
+constexpr uint32_t kIdescPV = kIdescBase | ((128u >> 3) << 17) | (1u << 16);    // N = D = 128
 
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   uint64_t d = 0;
@@ -54,25 +56,25 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= (uint64_t)2 << 61;   // 128-byte swizzle
   return d;
 }
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// A operand (16-bit, two K-elements per 32-bit column, one row per lane) read from TMEM
+// A operand (16-bit, two K-elements per 32-bit column, one row per lane) read from TMEM, B from shared memory
+// Called by ALL lanes of the (converged) MMA warp; one elected lane issues.  Keeping the warp converged lets
+// the compiler hold descriptors and addresses in uniform registers instead of serialising their arithmetic in
+// one divergent lane, which had limited the issue rate to about one MMA per 100 cycles.
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, e;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -93,22 +95,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
-        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])),
-        "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
-        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
-        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])),
-        "r"(__float_as_uint(v[31]))
-      : "memory");
-}
 __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -119,6 +105,12 @@ __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[3
         "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
         "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
       : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  uint32_t u[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) u[i] = __float_as_uint(v[i]);
+  tmem_st32u(taddr, u);
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -176,7 +168,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const int item_row0 = m_tile * kUmmaTileRows * 2;
   const int kv_begin = split * seg.chunk;
   const bool direct = seg.n_splits == 1;
-  // per 128-row tile: rows present, last key any of its rows sees, number of 128-key tiles to process
+  // per 128-row tile: rows present, last key any of its rows sees, number of 64-key tiles to process
   int t_rows[2], t_end[2], t_tiles[2], t_min_limit[2];
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
@@ -214,115 +206,125 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const uint32_t tmem = s_tmem_base;
   volatile int* abort_flag = &s_abort;
 
-  // register budget: the data-movement warpgroup gives registers to the two softmax warpgroups, which
-  // hold a whole 128-wide row of S per thread
+  // register budget: the data-movement warpgroup gives registers to the two softmax warpgroups
   if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-  if (warp == 8) {
-    // ================= producer: K0 V0 K1 V1 ... into the ring =================
-    if (n_tiles > 0) {
-      const int pages_per_tile = kTileKeys / g.S;
-      const int slab_block = g.S * 128;                      // bytes of one slab of a page block
-      const int copies = pages_per_tile * 2;                 // (page, slab) pairs per operand tile
-      for (int idx = 0; idx < 2 * n_tiles; ++idx) {
-        const int buf = idx % kNumBuf, use = idx / kNumBuf;
-        if (use > 0) mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status);
-        const int j = idx >> 1, is_v = idx & 1;
-        const int key0 = kv_begin + j * kTileKeys;
-        const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
-        const uint32_t bar = smem_u32(&bars.kv_full[buf]);
-        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * 2 * slab_block));
-        __syncwarp();
-        for (int c = lane; c < copies; c += 32) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 8) {
+      // ================= producer: K0 V0 K1 V1 ... into the ring =================
+      if (n_tiles > 0) {
+        const int pages_per_tile = kTileKeys / g.S;
+        const int slab_block = g.S * 128;                    // bytes of one slab of a page block
+        const int copies = pages_per_tile * 2;               // (page, slab) pairs per operand tile
+        // page ids are fetched 32 logical pages at a time, one per lane, a whole group ahead of their use,
+        // so that no bulk copy waits for a dependent page-table load
+        const int tiles_per_group = 32 / pages_per_tile;
+        const int lp0 = kv_begin / g.S;
+        const int32_t* trow = P.table + seg.table_off;
+        auto load_ids = [&](int grp) -> int {
+          const int lp = lp0 + grp * 32 + lane;
+          return lp < g.max_pages_per_task ? trow[lp] : 0;
+        };
+        int ids_cur = load_ids(0), ids_nxt = load_ids(1), cur_grp = 0;
+        for (int j = 0; j < n_tiles; ++j) {
+          const int buf = j % kNumBuf, use = j / kNumBuf;
+          const int grp = j / tiles_per_group;
+          if (grp != cur_grp) { ids_cur = ids_nxt; ids_nxt = load_ids(grp + 1); cur_grp = grp; }
+          if (use > 0) mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status);
+          const int key0 = kv_begin + j * kTileKeys;
+          const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
+          const uint32_t bar = smem_u32(&bars.kv_full[buf]);
+          if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * 4 * slab_block));
+          // lanes [0, copies) fetch the K pieces, lanes [copies, 2*copies) the V pieces of this tile
+          const int is_v = lane >= copies ? 1 : 0;
+          const int c = lane - is_v * copies;
           const int pg = c >> 1, slab = c & 1;
-          if (pg < npages) {
-            const long long page = P.table[seg.table_off + key0 / g.S + pg];
+          const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + pg) & 31);
+          if (lane < 2 * copies && pg < npages) {
             const uint8_t* src = P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes + is_v * g.kblock_bytes + slab * slab_block;
-            bulk_g2s(smem_base + kOffKV + buf * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
+            bulk_g2s(smem_base + buf * kSlotBytes + is_v * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
+          }
+        }
+        if (*abort_flag && lane == 0) {
+          // a wait gave up somewhere: do not leave while copies into this CTA's shared memory are in flight
+          for (int idx = max(0, n_tiles - kNumBuf); idx < n_tiles; ++idx) {
+            const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
+            const long long t0 = global_ns();
+            while (!mbar_try(bar, (idx / kNumBuf) & 1) && global_ns() - t0 < kWaitLimitNs) {}
           }
         }
       }
-      if (*abort_flag && lane == 0) {
-        for (int idx = max(0, 2 * n_tiles - kNumBuf); idx < 2 * n_tiles; ++idx) {
-          const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
-          const long long t0 = global_ns();
-          while (!mbar_try(bar, (idx / kNumBuf) & 1) && global_ns() - t0 < kWaitLimitNs) {}
-        }
-      }
-    }
-  } else if (warp == 9) {
-    // ================= MMA issuer (one lane) =================
-    if (lane == 0 && n_tiles > 0) {
-      TT_DECL;
-      mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
-      tc_fence_after();
-      auto issue_qk = [&](int t, int j) {
-        const int idx = 2 * j;
-        const uint32_t kbuf = smem_base + kOffKV + (idx % kNumBuf) * kTileBytes;
-        const uint32_t qbuf = smem_base + kOffQ + t * kTileBytes;
+    } else if (warp == 9) {
+      // ================= MMA issuer (whole warp converged, one elected lane issues) =================
+      if (n_tiles > 0) {
+        TT_DECL;
+        mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
+        tc_fence_after();
+        auto issue_qk = [&](int t, int j) {
+          const uint32_t kbuf = smem_base + (j % kNumBuf) * kSlotBytes;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
-          mma_ss(tmem + t * 128, make_desc(qbuf + off, 16, 1024), make_desc(kbuf + off, 16, 1024), kIdescQK, ks > 0);
-        }
-        mma_commit(smem_u32(&bars.s_full[t]));
-      };
-      auto issue_pv = [&](int t, int j) {
-        const int idx = 2 * j + 1;
-        const uint32_t vbuf = smem_base + kOffKV + (idx % kNumBuf) * kTileBytes;
+          for (int ks = 0; ks < D / 16; ++ks)
+            mma_ts(tmem + kColS + t * 64, tmem + kColQ + t * 64 + ks * 8,
+                   make_desc(kbuf + (ks >> 2) * kSlabBytes + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+          mma_commit(smem_u32(&bars.s_full[t]));
+        };
+        auto issue_pv = [&](int t, int j) {
+          const uint32_t vbuf = smem_base + (j % kNumBuf) * kSlotBytes + kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < kTileKeys / 16; ++ks)
-          mma_ts(tmem + 256 + t * 128, tmem + t * 128 + ks * 8, make_desc(vbuf + ks * 2048, kSlabBytes, 1024), kIdescPV,
-                 (j > 0 || ks > 0) ? 1u : 0u);
-      };
-      auto wait_full = [&](int idx) {
-        TT_BEGIN;
-        mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
-        TT_END(tt_wait2);
-      };
-      wait_full(0);
-      tc_fence_after();
-      for (int t = 0; t < 2; ++t) if (t_tiles[t] > 0) issue_qk(t, 0);
-      mma_commit(smem_u32(&bars.kv_empty[0]));
-      for (int j = 0; j < n_tiles; ++j) {
-        const int vidx = 2 * j + 1;
-        wait_full(vidx);
-        if (kv_end < kv_begin + (j + 1) * kTileKeys) {
-          // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
-          // them so that weight 0 times leftover bits cannot produce NaN
-          const int first = kv_end - (kv_begin + j * kTileKeys);
-          uint8_t* vgen = smem_gen + kOffKV + (vidx % kNumBuf) * kTileBytes;
-          for (int rr = first; rr < kTileKeys; ++rr)
-            for (int c = 0; c < 16; ++c)
+          for (int ks = 0; ks < kTileKeys / 16; ++ks)
+            mma_ts(tmem + kColO + t * 128, tmem + kColS + t * 64 + ks * 8, make_desc(vbuf + ks * 2048, kSlabBytes, 1024), kIdescPV,
+                   (j > 0 || ks > 0) ? 1u : 0u);
+        };
+        auto wait_full = [&](int idx) {
+          TT_BEGIN;
+          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+          TT_END(tt_wait2);
+        };
+        wait_full(0);
+        tc_fence_after();
+        for (int t = 0; t < 2; ++t) if (t_tiles[t] > 0) issue_qk(t, 0);
+        for (int j = 0; j < n_tiles; ++j) {
+          if (kv_end < kv_begin + (j + 1) * kTileKeys) {
+            // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
+            // them so that weight 0 times leftover bits cannot produce NaN
+            const int first = kv_end - (kv_begin + j * kTileKeys);
+            uint8_t* vgen = smem_gen + (j % kNumBuf) * kSlotBytes + kTileBytes;
+            for (int i = lane; i < (kTileKeys - first) * 16; i += 32) {
+              const int rr = first + (i >> 4), c = i & 15;
               *reinterpret_cast<uint4*>(vgen + (c >> 3) * kSlabBytes + rr * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
-          fence_async_smem();
-        }
-        const bool more = j + 1 < n_tiles;
-        if (more) wait_full(vidx + 1);
-        for (int t = 0; t < 2; ++t) {
-          if (j < t_tiles[t]) {
-            TT_BEGIN;
-            mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
-            TT_END(tt_wait);
-            tc_fence_after();
-            issue_pv(t, j);
-            if (j + 1 < t_tiles[t]) issue_qk(t, j + 1);             // overwrites S_t / P_t after PV_t(j), in order
-            else mma_commit(smem_u32(&bars.o_full[t]));
+            }
+            fence_async_smem();
+            __syncwarp();
           }
+          bool k_ready = false;
+          for (int t = 0; t < 2; ++t) {
+            if (j < t_tiles[t]) {
+              TT_BEGIN;
+              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
+              TT_END(tt_wait);
+              tc_fence_after();
+              issue_pv(t, j);
+              if (j + 1 < t_tiles[t]) {
+                if (!k_ready) { wait_full(j + 1); k_ready = true; }
+                issue_qk(t, j + 1);                          // overwrites S_t / P_t after PV_t(j), in order
+              } else {
+                mma_commit(smem_u32(&bars.o_full[t]));
+              }
+            }
+          }
+          mma_commit(smem_u32(&bars.kv_empty[j % kNumBuf]));   // K_j and V_j are consumed once PV(j) retires
         }
-        mma_commit(smem_u32(&bars.kv_empty[vidx % kNumBuf]));
-        if (more) mma_commit(smem_u32(&bars.kv_empty[(vidx + 1) % kNumBuf]));
+        // every MMA has completed (commits arrive in issue order) before this thread leaves
+        {
+          const int idx = n_tiles - 1;
+          mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+        }
+#ifdef TIDE_UMMA_TIMING
+        if (lane == 0) TT_FLUSH(2, 3, 4);
+#endif
       }
-      // every MMA has completed (commits arrive in issue order) before this thread leaves
-      {
-        const int idx = 2 * n_tiles - 1;
-        mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
-      }
-      TT_FLUSH(2, 3, 4);
     }
-  }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // ================= softmax warpgroups =================
     const int t = warp >> 2;                                   // 0 = A, 1 = B
     const int row = ((warp & 3) << 5) | lane;                  // row of the 128-row tile = TMEM lane
@@ -333,23 +335,28 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const int my_tiles = t_tiles[t];
     const int limit = valid ? min(t_end[t], seg.p + qi + 1) : t_end[t];   // keys j < limit are visible
 
-    // ---- stage this row of Q (or zeros) as an MMA operand ----
+    // ---- this row of Q (or zeros) into TMEM as the A operand of S = Q.K^T: two bf16 per column ----
     {
-      uint8_t* qrow = smem_gen + kOffQ + t * kTileBytes + row * 128;
       const uint4* src = reinterpret_cast<const uint4*>(P.q + ((long long)(seg.q_off + qi) * g.Hq + hd) * D);
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(qrow + (c >> 3) * kSlabBytes + (((c & 7) ^ (row & 7)) << 4)) = v;
+      for (int h = 0; h < 2; ++h) {
+        uint32_t qv[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 v = valid ? __ldg(src + h * 8 + c) : make_uint4(0, 0, 0, 0);
+          qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
+        }
+        tmem_st32u(tmem + lane_addr + kColQ + t * 64 + h * 32, qv);
       }
-      fence_async_smem();
+      tmem_wait_st();
+      tc_fence_before();
       mbar_arrive(smem_u32(&bars.q_full));
     }
 
     float m = -INFINITY, l = 0.f;       // running max (base-2, scaled) and sum
     const float sl2 = P.scale_log2e;
-    const uint32_t s_addr = tmem + lane_addr + t * 128;
-    const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
+    const uint32_t s_addr = tmem + lane_addr + kColS + t * 64;
+    const uint32_t o_addr = tmem + lane_addr + kColO + t * 128;
 
     TT_DECL;
     for (int j = 0; j < my_tiles; ++j) {
@@ -357,24 +364,24 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
       TT_END(tt_wait);
       tc_fence_after();
-      float s[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, *reinterpret_cast<float(*)[32]>(&s[c * 32]));
+      float s[64];
+      tmem_ld32(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
+      tmem_ld32(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_wait_ld();
       const int tile_key0 = kv_begin + j * kTileKeys;
       if (tile_key0 + kTileKeys > t_min_limit[t]) {            // uniform over the warpgroup
         const int vis = limit - tile_key0;
 #pragma unroll
-        for (int c = 0; c < 128; ++c) if (c >= vis) s[c] = -INFINITY;
+        for (int c = 0; c < 64; ++c) if (c >= vis) s[c] = -INFINITY;
       }
-      // independent partial reductions: a single 128-long dependent chain would expose its latency
+      // independent partial reductions: one long dependent chain would expose its latency
       float mxp[8];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) mxp[k] = fmaxf(s[k], s[k + 8]);
+      for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(s[i], s[i + 8]);
 #pragma unroll
-      for (int c = 16; c < 128; c += 16) {
+      for (int c = 16; c < 64; c += 16) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) mxp[k] = fmaxf(mxp[k], fmaxf(s[c + k], s[c + k + 8]));
+        for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(mxp[i], fmaxf(s[c + i], s[c + i + 8]));
       }
       float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
       mx *= sl2;                                               // scale > 0 on this path
@@ -396,22 +403,19 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       m = m_new;
       const float mu = (m == -INFINITY) ? 0.f : m;
       float sp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[32];
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t pk[32];
+      for (int c = 0; c < 64; c += 8) {
 #pragma unroll
-        for (int c = 0; c < 64; c += 8) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float e = fast_exp2(fmaf(s[h * 64 + c + k], sl2, -mu));
-            s[h * 64 + c + k] = e;
-            sp[k] += e;
-          }
-#pragma unroll
-          for (int k = 0; k < 4; ++k) pk[(c >> 1) + k] = pack_bf16(s[h * 64 + c + 2 * k], s[h * 64 + c + 2 * k + 1]);
+        for (int i = 0; i < 8; ++i) {
+          const float e = fast_exp2(fmaf(s[c + i], sl2, -mu));
+          s[c + i] = e;
+          sp[i] += e;
         }
-        tmem_st32u(s_addr + h * 32, pk);                       // P_t over the first 64 columns of S_t
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pk[(c >> 1) + i] = pack_bf16(s[c + 2 * i], s[c + 2 * i + 1]);
       }
+      tmem_st32u(s_addr, pk);                                  // P_t over the first 32 columns of S_t
       l = l * alpha + (((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7])));
       tmem_wait_st();
       tc_fence_before();
