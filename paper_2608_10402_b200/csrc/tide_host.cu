@@ -21,7 +21,7 @@ namespace {
 constexpr int kSlots = 4;                    // staging ring depth
 constexpr size_t kSlotPageIds = 64 * 1024;   // most new page ids per upload
 constexpr int kSlotRecs = 2048;              // most append records per upload
-constexpr int kTargetItemsPerSm = 8;
+constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
 constexpr int kNumSms = 148;
 constexpr long long kPartRowsBase = 256 * 1024;
 
@@ -74,6 +74,7 @@ struct tide_kv {
   cudaEvent_t ev_attend[4] = {nullptr, nullptr, nullptr, nullptr};
   bool have_append_times = false, have_attend_times = false;
   int umma_min_rows = kUmmaTileRows;  // packed rows from which a resume row takes the tcgen05 path
+  int items_per_sm = kTargetItemsPerSm;  // work items the planner aims for per SM
 };
 
 namespace {
@@ -227,6 +228,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->len.assign((size_t)cfg->max_tasks, 0);
   kv->pages.resize((size_t)cfg->max_tasks);
   kv->mark.assign((size_t)cfg->max_tasks, 0);
+  if (const char* e = getenv("TIDE_ITEMS_PER_SM")) kv->items_per_sm = std::max(1, atoi(e));  // tuning knob
   if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
   *out = kv;
@@ -489,7 +491,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
       else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
     }
   }
-  const long long target = (long long)kNumSms * kTargetItemsPerSm;
+  const long long target = (long long)kNumSms * kv->items_per_sm;
   long long chunk_dec = std::max<long long>(256, align_up((size_t)(w_dec / target + 1), kStageKeys));
   long long chunk_tile = (items_tile_nosplit >= target / 2)
                              ? (1LL << 30)
