@@ -28,8 +28,10 @@ __device__ __forceinline__ int chunk_offset(int S, int slot, int c) {
 constexpr int kAppendThreads = 256;
 constexpr int kAppendMaxRecsSmem = 1024;
 
-// One thread per 16-byte chunk of the source rows.  Chunks of a token are ordered [K|V][kv_head][c], so a
-// warp reads 512 contiguous source bytes and writes four full 128-byte lines.
+// One warp per token at a time: the record lookup, the page-table read and the slot arithmetic happen once per
+// token (warp-uniform), then the lanes copy the token's 16-byte chunks, ordered [K|V][kv_head][chunk], so a warp
+// reads 512 contiguous source bytes and writes four full 128-byte lines per pass.  D/8 is a power of two, so the
+// per-chunk index split needs no division.
 __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const AppendParams P) {
   __shared__ int32_t s_tok0[kAppendMaxRecsSmem];
   const int n_recs = P.n_recs;
@@ -38,17 +40,13 @@ __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const Ap
     for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = P.recs[i].tok0;
     __syncthreads();
   }
-  const int cpr = P.g.D >> 3;                 // chunks per (token, head) row
-  const int cpt = 2 * P.g.Hkv * cpr;          // chunks per token, K and V
-  const long long total = (long long)P.n_tokens * cpt;
-  for (long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x; gid < total;
-       gid += (long long)gridDim.x * blockDim.x) {
-    const int tok = (int)(gid / cpt);
-    int rem = (int)(gid - (long long)tok * cpt);
-    const int kv = rem / (P.g.Hkv * cpr);
-    rem -= kv * P.g.Hkv * cpr;
-    const int h = rem / cpr;
-    const int c = rem - h * cpr;
+  const int lane = threadIdx.x & 31;
+  const int cpr = P.g.D >> 3;                 // chunks per (token, head) row: 8 or 16
+  const int shift = cpr == 16 ? 4 : 3;
+  const int rows2 = 2 * P.g.Hkv;              // K rows then V rows of one token
+  const int cpt = rows2 * cpr;                // chunks per token
+  const int warps_total = gridDim.x * (kAppendThreads / 32);
+  for (int tok = blockIdx.x * (kAppendThreads / 32) + (threadIdx.x >> 5); tok < P.n_tokens; tok += warps_total) {
     int r;
     if (in_smem) r = find_segment(n_recs, tok, [&](int i) { return s_tok0[i]; });
     else r = find_segment(n_recs, tok, [&](int i) { return P.recs[i].tok0; });
@@ -56,18 +54,27 @@ __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const Ap
     const int pos = rec.pos0 + (tok - rec.tok0);
     const int lp = pos / P.g.S, slot = pos - lp * P.g.S;
     const long long page = P.table[rec.table_off + lp];
-    const uint16_t* src = (kv ? P.new_v : P.new_k) + ((long long)tok * P.g.Hkv + h) * P.g.D + c * 8;
-    uint8_t* dst = P.pool + page * P.g.page_bytes + (long long)h * P.g.head_bytes + kv * P.g.kblock_bytes +
-                   chunk_offset(P.g.S, slot, c);
-    *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    uint8_t* page_base = P.pool + page * P.g.page_bytes + slot * 128;
+    const uint16_t* src_k = P.new_k + (long long)tok * P.g.Hkv * P.g.D;
+    const uint16_t* src_v = P.new_v + (long long)tok * P.g.Hkv * P.g.D;
+    const int sw = slot & 7;
+    for (int c = lane; c < cpt; c += 32) {
+      const int cc = c & (cpr - 1);
+      const int row = c >> shift;               // 0 .. 2*Hkv-1
+      const int kv = row >= P.g.Hkv ? 1 : 0;
+      const int h = row - kv * P.g.Hkv;
+      const uint16_t* src = (kv ? src_v : src_k) + h * P.g.D + cc * 8;
+      uint8_t* dst = page_base + (long long)h * P.g.head_bytes + kv * P.g.kblock_bytes + (cc >> 3) * (P.g.S * 128) +
+                     (((cc & 7) ^ sw) << 4);
+      *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    }
   }
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
   if (p.n_tokens <= 0) return cudaSuccess;
-  const long long total = (long long)p.n_tokens * 2 * p.g.Hkv * (p.g.D / 8);
-  long long blocks = (total + kAppendThreads - 1) / kAppendThreads;
-  const long long cap = 148LL * 8 * 16;  // grid-stride beyond this
+  long long blocks = ((long long)p.n_tokens + kAppendThreads / 32 - 1) / (kAppendThreads / 32);
+  const long long cap = 148LL * 8 * 8;   // 8 resident blocks per SM, a few tokens per warp beyond this
   if (blocks > cap) blocks = cap;
   append_scatter_kernel<<<(unsigned)blocks, kAppendThreads, 0, s>>>(p);
   return cudaGetLastError();
