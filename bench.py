@@ -30,8 +30,8 @@ METRIC = "mixed resume batch: KV-read GB/s vs HBM peak; append-prefill TFLOP/s v
 # DRAM traffic per unit of algorithmic work, from the ncu captures summarised under profiles/ (reduced cases,
 # scaled by the units one launch processes): decode kernel dram bytes / algorithmic KV bytes; tcgen05 kernel
 # dram bytes per flop of resume-row attention.
-NCU_DECODE_TRAFFIC_RATIO = 1.014
-NCU_UMMA_DRAM_BYTES_PER_FLOP = 96.4e6 / 191.7e9
+NCU_DECODE_TRAFFIC_RATIO = 1.011
+NCU_UMMA_DRAM_BYTES_PER_FLOP = 349.7e6 / 863.8e9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -229,7 +229,7 @@ def run_ours(args):
         roof_tensor = {"bound": "tensor", "kernel": "attend tile kernel (resume rows)",
                        "achieved": res_flops / (ph_ms["tile"] * 1e-3) / 1e12 if ph_ms["tile"] > 0 else 0.0,
                        "peak": tpeak, "unit": "TFLOP/s", "traffic": res_flops * NCU_UMMA_DRAM_BYTES_PER_FLOP,
-                       "traffic_note": "dram read bytes of a reduced-case ncu capture scaled by flops (see profiles/)",
+                       "traffic_note": "dram read+write bytes of a reduced-case ncu capture scaled by flops (see profiles/)",
                        "peak_source": f"{peaks['_source']} ({'sustained' if sustained else 'burst'} bf16)"}
         roof_tensor["frac"] = roof_tensor["achieved"] / tpeak
         roof_hbm = {"bound": "hbm", "kernel": "attend decode kernel (decode rows)",
