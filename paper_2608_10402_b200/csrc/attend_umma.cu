@@ -185,6 +185,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const int n_tiles = max(t_tiles[0], t_tiles[1]);
   const int kv_end = max(t_end[0], t_end[1]);
 
+  // a bounded wait that ran out in an earlier CTA of this launch means something is wrong: start no more work
+  __shared__ int s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int*>(P.status);
+  __syncthreads();
+  if (s_skip != 0) return;
+
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
@@ -206,7 +212,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const uint32_t tmem = s_tmem_base;
   volatile int* abort_flag = &s_abort;
 
-  // register budget: the data-movement warpgroup gives registers to the two softmax warpgroups
+  // register budget: the data-movement warpgroup gives registers to the two softmax warpgroups.  setmaxnreg
+  // moves registers inside the CTA's own launch allocation (384 x 168), so the new counts must not add up to
+  // more than that: 256 x 224 + 128 x 56 = 384 x 168.  (An over-subscribed .inc waits for ever.)
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 8) {
