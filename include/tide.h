@@ -137,6 +137,17 @@ int tide_kv_release(tide_kv_t* kv, int32_t task);
  * (sliding-window pruning of old observations, Appendix C.2).  Host only. */
 int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len);
 
+/* tide_kv_release for several tasks at once (a finished GRPO group, or every task a scheduler evicts in one
+ * pass of Algorithm 1).  All-or-nothing: unknown or repeated ids release nothing. */
+int tide_kv_release_many(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids /*host*/);
+
+/* Sliding-window pruning of old observations (Appendix C.2: only the most recent images are kept, which splits
+ * the trajectory): the task keeps tokens [0, keep_prefix) and [tail_begin, len); the tokens in between are
+ * dropped and the tail moves down to start at keep_prefix.  Equivalent, page table included, to reading the
+ * tail, tide_kv_truncate(task, keep_prefix) and appending the tail again; the move runs on `stream` through
+ * the workspace staging area.  Requires 0 <= keep_prefix <= tail_begin <= len. */
+int tide_kv_prune(tide_kv_t* kv, int32_t layer, int32_t task, int32_t keep_prefix, int32_t tail_begin, void* stream);
+
 /* Introspection (the per-rank token usage CTB schedules on, Section 4.1 / Algorithm 1). */
 int tide_kv_task_len(tide_kv_t* kv, int32_t task, int32_t* len);
 int tide_kv_page_table(tide_kv_t* kv, int32_t task, int32_t* out /*host*/, int32_t cap, int32_t* n_pages);

@@ -178,6 +178,33 @@ class PagedKVOracle:
             self.free.append(self.pages[task].pop())
         self.len[task] = new_len
 
+    def release_many(self, tasks):
+        tasks = [int(t) for t in tasks]
+        for t in tasks:
+            self._check_live(t)
+        if len(set(tasks)) != len(tasks):
+            raise OracleError(ERR_DUPLICATE_TASK, "a task appears twice")
+        for t in tasks:
+            self.release(t)
+
+    def prune(self, task: int, keep_prefix: int, tail_begin: int):
+        """Sliding-window pruning (Appendix C.2): keep tokens [0, keep_prefix) and [tail_begin, len), written
+        out as its definition: read the tail, truncate to keep_prefix, append the tail again."""
+        self._check_live(task)
+        if not (0 <= keep_prefix <= tail_begin <= self.len[task]):
+            raise OracleError(ERR_INVALID_ARG, "need 0 <= keep_prefix <= tail_begin <= len")
+        if keep_prefix == tail_begin:
+            return
+        if self.store_values:
+            k, v = self.read(task)
+            tail_k, tail_v = k[tail_begin:].copy(), v[tail_begin:].copy()
+        n_tail = self.len[task] - tail_begin
+        self.truncate(task, keep_prefix)
+        if self.store_values:
+            self.append([task], [0, n_tail], tail_k, tail_v)
+        else:
+            self.append([task], [0, n_tail])
+
     def reset(self, free_order=None):
         """Flush every task (the cache flush at a weight synchronisation,
         Section 5.2) and restart the free stack from free_order."""

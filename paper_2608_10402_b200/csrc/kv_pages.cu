@@ -81,35 +81,37 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
 }
 
 // Logical content of one task -> contiguous [len, Hkv, D]; inverse of the scatter above.
-__global__ void read_gather_kernel(const uint8_t* __restrict__ pool, const int32_t* __restrict__ table_row, int len,
+// Positions [pos0, pos0 + len) of the task go to rows [0, len) of out_k / out_v.
+__global__ void read_gather_kernel(const uint8_t* __restrict__ pool, const int32_t* __restrict__ table_row, int pos0, int len,
                                    uint16_t* __restrict__ out_k, uint16_t* __restrict__ out_v, const Geom g) {
   const int cpr = g.D >> 3;
   const int cpt = 2 * g.Hkv * cpr;
   const long long total = (long long)len * cpt;
   for (long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x; gid < total;
        gid += (long long)gridDim.x * blockDim.x) {
-    const int pos = (int)(gid / cpt);
-    int rem = (int)(gid - (long long)pos * cpt);
+    const int row = (int)(gid / cpt);
+    int rem = (int)(gid - (long long)row * cpt);
     const int kv = rem / (g.Hkv * cpr);
     rem -= kv * g.Hkv * cpr;
     const int h = rem / cpr;
     const int c = rem - h * cpr;
+    const int pos = pos0 + row;
     const int lp = pos / g.S, slot = pos - lp * g.S;
     const long long page = table_row[lp];
     const uint8_t* src = pool + page * g.page_bytes + (long long)h * g.head_bytes + kv * g.kblock_bytes +
                          chunk_offset(g.S, slot, c);
-    uint16_t* dst = (kv ? out_v : out_k) + ((long long)pos * g.Hkv + h) * g.D + c * 8;
+    uint16_t* dst = (kv ? out_v : out_k) + ((long long)row * g.Hkv + h) * g.D + c * 8;
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
 }
 
-cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int len, uint16_t* out_k, uint16_t* out_v,
-                        const Geom& g, cudaStream_t s) {
+cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int pos0, int len, uint16_t* out_k,
+                        uint16_t* out_v, const Geom& g, cudaStream_t s) {
   if (len <= 0) return cudaSuccess;
   const long long total = (long long)len * 2 * g.Hkv * (g.D / 8);
   long long blocks = (total + 255) / 256;
   if (blocks > 148LL * 64) blocks = 148LL * 64;
-  read_gather_kernel<<<(unsigned)blocks, 256, 0, s>>>(pool, table_row, len, out_k, out_v, g);
+  read_gather_kernel<<<(unsigned)blocks, 256, 0, s>>>(pool, table_row, pos0, len, out_k, out_v, g);
   return cudaGetLastError();
 }
 

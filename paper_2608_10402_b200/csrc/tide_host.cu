@@ -449,8 +449,54 @@ int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k, void* 
   if (kv->len[task] == 0) return TIDE_OK;
   if (out_k == nullptr || out_v == nullptr || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15)) return TIDE_ERR_INVALID_ARG;
   const int32_t* row = kv->d_table + (size_t)task * kv->g.max_pages_per_task;
-  if (launch_read(kv->pool, row, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
+  if (launch_read(kv->pool, row, 0, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
     return TIDE_ERR_CUDA;
+  return TIDE_OK;
+}
+
+int tide_kv_release_many(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids) {
+  if (kv == nullptr || n_tasks < 0 || (n_tasks > 0 && task_ids == nullptr)) return TIDE_ERR_INVALID_ARG;
+  for (int j = 0; j < n_tasks; ++j) {
+    if (!task_in_range(kv, task_ids[j])) return TIDE_ERR_INVALID_ARG;
+    if (!kv->live[task_ids[j]]) return TIDE_ERR_UNKNOWN_TASK;
+  }
+  if (++kv->mark_gen == 0x7fffffff) {
+    std::fill(kv->mark.begin(), kv->mark.end(), 0);
+    kv->mark_gen = 1;
+  }
+  for (int j = 0; j < n_tasks; ++j) {
+    if (kv->mark[task_ids[j]] == kv->mark_gen) return TIDE_ERR_DUPLICATE_TASK;
+    kv->mark[task_ids[j]] = kv->mark_gen;
+  }
+  for (int j = 0; j < n_tasks; ++j) tide_kv_release(kv, task_ids[j]);
+  return TIDE_OK;
+}
+
+int tide_kv_prune(tide_kv_t* kv, int32_t layer, int32_t task, int32_t keep_prefix, int32_t tail_begin, void* stream) {
+  if (kv == nullptr || layer != 0 || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  const int len = kv->len[task];
+  if (!(0 <= keep_prefix && keep_prefix <= tail_begin && tail_begin <= len)) return TIDE_ERR_INVALID_ARG;
+  const int tail = len - tail_begin;
+  if (tail_begin == keep_prefix) return TIDE_OK;   // nothing is dropped
+  const Geom& g = kv->g;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint16_t* sk = (uint16_t*)(kv->ws + kv->lay.off_stage_k);
+  uint16_t* sv = (uint16_t*)(kv->ws + kv->lay.off_stage_v);
+  const int chunk_cap = (int)std::min<int64_t>(kv->cfg.max_batch_tokens, 0x7fffffff);
+  // The shorter task needs no more pages than it holds, and truncate returns pages in the order in which the
+  // appends below take them again, so the kept part of the table does not change and nothing can fail below.
+  int rc = tide_kv_truncate(kv, task, keep_prefix);
+  if (rc != TIDE_OK) return rc;
+  const int32_t* row = kv->d_table + (size_t)task * g.max_pages_per_task;
+  // Move the tail down in chunks, front to back: a chunk is written below the positions the next one reads.
+  for (int done = 0; done < tail; done += chunk_cap) {
+    const int n = std::min(chunk_cap, tail - done);
+    if (launch_read(kv->pool, row, tail_begin + done, n, sk, sv, g, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    const int32_t ip[2] = {0, n};
+    rc = tide_kv_append(kv, layer, 1, &task, ip, sk, sv, stream);
+    if (rc != TIDE_OK) return rc;
+  }
   return TIDE_OK;
 }
 

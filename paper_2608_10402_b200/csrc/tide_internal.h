@@ -94,8 +94,8 @@ struct AppendParams {
 
 cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s);
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s);
-cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int len, uint16_t* out_k, uint16_t* out_v,
-                        const Geom& g, cudaStream_t s);
+cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int pos0, int len, uint16_t* out_k,
+                        uint16_t* out_v, const Geom& g, cudaStream_t s);
 cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s);
 cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);

@@ -46,7 +46,7 @@ EXPORTS = [
     "tide_strerror", "tide_kv_required_bytes", "tide_kv_create", "tide_kv_destroy", "tide_kv_reset",
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
-    "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static",
+    "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -157,6 +157,14 @@ class TideKV:
 
     def release(self, task):
         _check(lib.tide_kv_release(self.handle, ctypes.c_int32(task)), "tide_kv_release")
+
+    def release_many(self, task_ids):
+        ids = _i32(task_ids)
+        _check(lib.tide_kv_release_many(self.handle, ctypes.c_int32(ids.shape[0]), _ptr(ids)), "tide_kv_release_many")
+
+    def prune(self, task, keep_prefix, tail_begin, stream=None):
+        _check(lib.tide_kv_prune(self.handle, ctypes.c_int32(0), ctypes.c_int32(task), ctypes.c_int32(keep_prefix),
+                                 ctypes.c_int32(tail_begin), _stream(stream)), "tide_kv_prune")
 
     def truncate(self, task, new_len):
         _check(lib.tide_kv_truncate(self.handle, ctypes.c_int32(task), ctypes.c_int32(new_len)), "tide_kv_truncate")

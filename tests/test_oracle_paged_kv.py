@@ -211,3 +211,37 @@ def test_every_error_leaves_state_unchanged():
     c.alloc(2, reserve_tokens=8)   # exactly the headroom: admitted
     c.append([1], [0, 0], z[:0], z[:0])  # zero-length append is a no-op
     assert c.task_len(1) == 0 and list(c.page_table(1)) == []
+
+
+def test_prune_keeps_prefix_and_tail_and_reuses_pages():
+    # sliding-window pruning: tokens [0, keep) and [tail_begin, len) survive, in order, and the task ends up with
+    # exactly the pages a task of the new length needs, the first of them unchanged
+    rng = np.random.default_rng(17)
+    c = PagedKVOracle(20, 4, 2, 4, 3, 12, free_order=rng.permutation(20))
+    k = rng.integers(0, 65536, size=(30, 2, 4)).astype(np.uint16)
+    v = rng.integers(0, 65536, size=(30, 2, 4)).astype(np.uint16)
+    c.alloc(0)
+    c.alloc(1)
+    c.append([0], [0, 30], k, v)
+    c.append([1], [0, 5], k[:5], v[:5])
+    before = list(c.page_table(0))
+    free_before = c.free_pages()
+    c.prune(0, 6, 17)                      # drop positions 6..16
+    gk, gv = c.read(0)
+    assert c.task_len(0) == 6 + 13
+    assert np.array_equal(gk, np.concatenate([k[:6], k[17:]])) and np.array_equal(gv, np.concatenate([v[:6], v[17:]]))
+    assert list(c.page_table(0)) == before[:5]          # ceil(19 / 4) = 5 pages, the same ones in the same order
+    assert c.free_pages() == free_before + 3
+    assert np.array_equal(c.read(1)[0], k[:5])          # the neighbour is untouched
+    c.prune(0, 19, 19)                                  # nothing dropped: no-op
+    assert c.task_len(0) == 19
+    c.prune(0, 0, 19)                                   # everything dropped
+    assert c.task_len(0) == 0 and list(c.page_table(0)) == []
+    with pytest.raises(OracleError):
+        c.prune(1, 3, 2)
+    c.release_many([0, 1])
+    assert c.free_pages() == 20 and not c.live
+    c.alloc(2)
+    with pytest.raises(OracleError) as e:
+        c.release_many([2, 2])
+    assert e.value.code == pk.ERR_DUPLICATE_TASK and 2 in c.live
