@@ -84,6 +84,12 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
     return;
   }
 
+  // a bounded wait that ran out in an earlier CTA of this launch means something is wrong: start no more work
+  __shared__ int s_skip;
+  if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int*>(P.status);
+  __syncthreads();
+  if (s_skip != 0) return;
+
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int i = 0; i < kStages; ++i) {
