@@ -137,6 +137,18 @@ int tide_kv_release(tide_kv_t* kv, int32_t task);
  * (sliding-window pruning of old observations, Appendix C.2).  Host only. */
 int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len);
 
+/* Group-shared prefixes (a GRPO group rolls out G trajectories from one prompt, Section 2.1; CTB's worker
+ * affinity keeps a group on the rank that holds its shared prefix, end of Section 4).  `child` becomes a live
+ * task whose content is the parent's current content: the parent's full pages are SHARED (reference counted,
+ * never written again), a partial last page is copied into a fresh page, so parent and child can both keep
+ * appending.  A page returns to the free stack when its last holder lets go of it.  An append that would write
+ * into a page other tasks still hold (possible after tide_kv_truncate into shared pages) first replaces it by
+ * a private copy, taken from the free stack before the task's other new pages.  Errors: TIDE_ERR_TASK_EXISTS,
+ * TIDE_ERR_UNKNOWN_TASK, TIDE_ERR_NO_PAGES (no page for the copy). */
+int tide_kv_fork(tide_kv_t* kv, int32_t layer, int32_t parent, int32_t child, void* stream);
+/* How many tasks hold each page of `task` (same order as tide_kv_page_table). */
+int tide_kv_page_refs(tide_kv_t* kv, int32_t task, int32_t* out /*host*/, int32_t cap, int32_t* n_pages);
+
 /* tide_kv_release for several tasks at once (a finished GRPO group, or every task a scheduler evicts in one
  * pass of Algorithm 1).  All-or-nothing: unknown or repeated ids release nothing. */
 int tide_kv_release_many(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids /*host*/);

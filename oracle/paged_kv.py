@@ -17,6 +17,15 @@ that page tables can be compared bit for bit:
   * release pushes a task's pages back last-to-first, so re-appending the same
     length straight away receives the same pages in the same order
   * truncate(task, new_len) pushes back pages ceil(new_len/S).. last-to-first
+  * pages are reference counted so that the trajectories of a GRPO group can
+    share their common prefix (Section 2.1: G trajectories per prompt; end of
+    Section 4: worker affinity keeps shared prefixes on one rank).
+    fork(parent, child) gives the child the parent's FULL pages (count + 1
+    each) and a fresh copy of the parent's partial last page, if any; a page
+    goes back to the free stack only when its count drops to 0; an append that
+    would write into a page whose count is above 1 (possible after a truncate
+    into shared pages) first replaces it by a private copy, popped before the
+    task's other pages
 
 Cache contents are raw bf16 bit patterns (uint16); this module never does
 floating-point arithmetic.  Physical storage here is token-major
@@ -69,6 +78,7 @@ class PagedKVOracle:
         self.live = {}          # task -> True
         self.len = {}           # task -> resident tokens
         self.pages = {}         # task -> list of physical pages
+        self.ref = {}           # physical page -> number of tasks holding it (absent = free)
         self.store_values = store_values
         if store_values:
             self.pool_k = np.zeros((self.P, self.S, self.Hkv, self.D), dtype=np.uint16)
@@ -94,7 +104,8 @@ class PagedKVOracle:
 
     def state_hash(self):
         """A value that changes whenever any bookkeeping changes."""
-        return (tuple(self.free), tuple(sorted((t, self.len[t], tuple(self.pages[t])) for t in self.live)))
+        return (tuple(self.free), tuple(sorted((t, self.len[t], tuple(self.pages[t])) for t in self.live)),
+                tuple(sorted(self.ref.items())))
 
     def _check_task_id(self, task: int):
         if not (0 <= task < self.max_tasks):
@@ -147,26 +158,81 @@ class PagedKVOracle:
             c = indptr[j + 1] - indptr[j]
             after = _ceil_div(self.len[t] + c, self.S)
             need_total += after - _ceil_div(self.len[t], self.S)
+            if c > 0 and self._last_page_is_shared(t):
+                need_total += 1
             if after > self.max_pages_per_task:
                 raise OracleError(ERR_TABLE_FULL, f"task {t} would need {after} pages")
         if need_total > len(self.free):
             raise OracleError(ERR_NO_PAGES, f"need {need_total} pages, {len(self.free)} free")
         # ---- mutation starts here ----
         for j, t in enumerate(task_ids):
+            if indptr[j + 1] > indptr[j] and self._last_page_is_shared(t):
+                self._make_last_page_private(t)
             for i in range(indptr[j + 1] - indptr[j]):
                 pos = self.len[t] + i
                 if pos % self.S == 0:
-                    self.pages[t].append(self.free.pop())
+                    self.pages[t].append(self._pop())
                 if self.store_values:
                     page, slot = self.pages[t][pos // self.S], pos % self.S
                     self.pool_k[page, slot] = new_k[indptr[j] + i]
                     self.pool_v[page, slot] = new_v[indptr[j] + i]
             self.len[t] += indptr[j + 1] - indptr[j]
 
+    # ---- reference counting ---------------------------------------------
+    def _pop(self) -> int:
+        page = self.free.pop()
+        self.ref[page] = 1
+        return page
+
+    def _unref(self, page: int):
+        self.ref[page] -= 1
+        if self.ref[page] == 0:
+            del self.ref[page]
+            self.free.append(page)
+
+    def _last_page_is_shared(self, task: int) -> bool:
+        return self.len[task] % self.S != 0 and self.ref[self.pages[task][-1]] > 1
+
+    def _make_last_page_private(self, task: int):
+        old = self.pages[task][-1]
+        new = self._pop()
+        if self.store_values:
+            self.pool_k[new] = self.pool_k[old]
+            self.pool_v[new] = self.pool_v[old]
+        self.pages[task][-1] = new
+        self._unref(old)
+
+    def fork(self, parent: int, child: int):
+        """child becomes a live task with the parent's current content; full pages are shared."""
+        self._check_live(parent)
+        self._check_task_id(child)
+        if child in self.live:
+            raise OracleError(ERR_TASK_EXISTS, f"task {child} already live")
+        L = self.len[parent]
+        n_full = L // self.S
+        if L % self.S and not self.free:
+            raise OracleError(ERR_NO_PAGES, "no page for the copy of the partial last page")
+        self.live[child] = True
+        self.len[child] = L
+        self.pages[child] = list(self.pages[parent][:n_full])
+        for page in self.pages[child]:
+            self.ref[page] += 1
+        if L % self.S:
+            new = self._pop()
+            if self.store_values:
+                old = self.pages[parent][n_full]
+                self.pool_k[new] = self.pool_k[old]
+                self.pool_v[new] = self.pool_v[old]
+            self.pages[child].append(new)
+
+    def page_refs(self, task: int) -> np.ndarray:
+        self._check_live(task)
+        return np.asarray([self.ref[p] for p in self.pages[task]], dtype=np.int32)
+
     def release(self, task: int):
         self._check_live(task)
         for page in reversed(self.pages[task]):
-            self.free.append(page)
+            self._unref(page)
         del self.live[task], self.len[task], self.pages[task]
 
     def truncate(self, task: int, new_len: int):
@@ -175,7 +241,7 @@ class PagedKVOracle:
             raise OracleError(ERR_INVALID_ARG, "new_len outside [0, len]")
         keep = _ceil_div(new_len, self.S)
         while len(self.pages[task]) > keep:
-            self.free.append(self.pages[task].pop())
+            self._unref(self.pages[task].pop())
         self.len[task] = new_len
 
     def release_many(self, tasks):
@@ -214,7 +280,7 @@ class PagedKVOracle:
         if free_order.shape != (self.P,) or not np.array_equal(np.sort(free_order), np.arange(self.P)):
             raise OracleError(ERR_INVALID_ARG, "free_order is not a permutation")
         self.free = [int(p) for p in free_order[::-1]]
-        self.live, self.len, self.pages = {}, {}, {}
+        self.live, self.len, self.pages, self.ref = {}, {}, {}, {}
 
     # ---- reads -----------------------------------------------------------
     def read(self, task: int, length=None):

@@ -80,6 +80,23 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+// Whole-page copies dst[i] <- src[i] (the private copy a forked task gets of a partial last page, and the copy an
+// append makes before it writes into a page that other tasks still hold).  One block column per page.
+__global__ void copy_pages_kernel(uint8_t* __restrict__ pool, const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
+                                  long long page_bytes) {
+  const uint4* s = reinterpret_cast<const uint4*>(pool + (long long)src[blockIdx.y] * page_bytes);
+  uint4* d = reinterpret_cast<uint4*>(pool + (long long)dst[blockIdx.y] * page_bytes);
+  const long long n = page_bytes / 16;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) d[i] = s[i];
+}
+
+cudaError_t launch_copy_pages(uint8_t* pool, const int32_t* src, const int32_t* dst, int n, long long page_bytes, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  dim3 grid(8, (unsigned)n);
+  copy_pages_kernel<<<grid, 256, 0, s>>>(pool, src, dst, page_bytes);
+  return cudaGetLastError();
+}
+
 // Logical content of one task -> contiguous [len, Hkv, D]; inverse of the scatter above.
 // Positions [pos0, pos0 + len) of the task go to rows [0, len) of out_k / out_v.
 __global__ void read_gather_kernel(const uint8_t* __restrict__ pool, const int32_t* __restrict__ table_row, int pos0, int len,

@@ -62,6 +62,7 @@ struct tide_kv {
   std::vector<uint8_t> live;
   std::vector<int32_t> len;
   std::vector<std::vector<int32_t>> pages;
+  std::vector<int32_t> refcnt;  // per physical page: how many tasks hold it (0 = free)
   std::vector<int32_t> mark;  // scratch for duplicate detection
   int32_t mark_gen = 0;
   int64_t used_tokens = 0;
@@ -108,7 +109,7 @@ Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
   size_t off = 0;
   L.off_status = off; off += 256;
   L.off_table = off; off = align_up(off + (size_t)c->max_tasks * c->max_pages_per_task * 4, 256);
-  L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 +
+  L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 + (size_t)kSlotRecs * 8 +
                               (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
   L.off_meta = off; off += L.slot_bytes * kSlots;
   L.part_rows = kPartRowsBase + (long long)g.Hq * c->max_batch_rows * 4;
@@ -142,6 +143,23 @@ void prime_free_stack(tide_kv* kv, const int32_t* order) {
 }
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+int32_t pop_page(tide_kv* kv) {
+  const int32_t page = kv->free_stack.back();
+  kv->free_stack.pop_back();
+  kv->refcnt[(size_t)page] = 1;
+  return page;
+}
+
+// Drops one holder of `page`; the page returns to the free stack when nobody holds it any more.
+void unref_page(tide_kv* kv, int32_t page) {
+  if (--kv->refcnt[(size_t)page] == 0) kv->free_stack.push_back(page);
+}
+
+// True if the next token of `task` would be written into a page that another task also holds.
+bool last_page_shared(const tide_kv* kv, int32_t task) {
+  return kv->len[task] % kv->g.S != 0 && kv->refcnt[(size_t)kv->pages[task].back()] > 1;
+}
 
 bool task_in_range(const tide_kv* kv, int32_t t) { return t >= 0 && t < kv->cfg.max_tasks; }
 
@@ -228,6 +246,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->len.assign((size_t)cfg->max_tasks, 0);
   kv->pages.resize((size_t)cfg->max_tasks);
   kv->mark.assign((size_t)cfg->max_tasks, 0);
+  kv->refcnt.assign((size_t)cfg->num_pages, 0);
   if (const char* e = getenv("TIDE_ITEMS_PER_SM")) kv->items_per_sm = std::max(1, atoi(e));  // tuning knob
   if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
@@ -256,6 +275,7 @@ int tide_kv_reset(tide_kv_t* kv, const int32_t* free_order) {
   std::fill(kv->live.begin(), kv->live.end(), 0);
   std::fill(kv->len.begin(), kv->len.end(), 0);
   for (auto& p : kv->pages) p.clear();
+  std::fill(kv->refcnt.begin(), kv->refcnt.end(), 0);
   kv->used_tokens = 0;
   prime_free_stack(kv, free_order);
   return TIDE_OK;
@@ -275,7 +295,7 @@ int tide_kv_release(tide_kv_t* kv, int32_t task) {
   if (kv == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
   if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
   auto& pg = kv->pages[task];
-  for (size_t i = pg.size(); i-- > 0;) kv->free_stack.push_back(pg[i]);
+  for (size_t i = pg.size(); i-- > 0;) unref_page(kv, pg[i]);
   pg.clear();
   kv->used_tokens -= kv->len[task];
   kv->len[task] = 0;
@@ -290,7 +310,7 @@ int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len) {
   auto& pg = kv->pages[task];
   const size_t keep = (size_t)ceil_div(new_len, kv->g.S);
   while (pg.size() > keep) {
-    kv->free_stack.push_back(pg.back());
+    unref_page(kv, pg.back());
     pg.pop_back();
   }
   kv->used_tokens -= kv->len[task] - new_len;
@@ -354,6 +374,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
     const int after = ceil_div(kv->len[t] + c, g.S);
     if (after > g.max_pages_per_task) return TIDE_ERR_TABLE_FULL;
     need += after - ceil_div(kv->len[t], g.S);
+    if (c > 0 && last_page_shared(kv, t)) ++need;   // a private copy of the shared partial page comes first
   }
   if (need > (long long)kv->free_stack.size()) return TIDE_ERR_NO_PAGES;
 
@@ -369,7 +390,9 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
     AppendRec* recs = (AppendRec*)(slot->host + 256);
     int32_t* idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
     int32_t* val = idx + kSlotPageIds;
-    int n_recs = 0;
+    int32_t* cpy_src = val + kSlotPageIds;
+    int32_t* cpy_dst = cpy_src + kSlotRecs;
+    int n_recs = 0, n_cpy = 0;
     size_t n_ids = 0;
     int tok_lo = -1, tok_hi = -1;
     while (j < n_tasks && n_recs < kSlotRecs) {
@@ -377,6 +400,20 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
       const int c = indptr[j + 1] - indptr[j];
       int remaining = c - done_in_task;
       if (remaining == 0) { ++j; done_in_task = 0; continue; }
+      if (done_in_task == 0 && last_page_shared(kv, t)) {
+        // the task ends inside a page that others hold: give it a private copy before anything is written
+        if (n_ids == kSlotPageIds) break;
+        auto& pg0 = kv->pages[t];
+        const int32_t old_page = pg0.back(), new_page = pop_page(kv);
+        cpy_src[n_cpy] = old_page;
+        cpy_dst[n_cpy] = new_page;
+        ++n_cpy;
+        idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg0.size() - 1;
+        val[n_ids] = new_page;
+        ++n_ids;
+        pg0.back() = new_page;
+        unref_page(kv, old_page);
+      }
       const int pos0 = kv->len[t];
       // tokens that fit: up to the page-id budget of this upload
       const int room_in_last = (int)((long long)ceil_div(pos0, g.S) * g.S - pos0);
@@ -387,8 +424,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
       const int new_pages = ceil_div(pos0 + take, g.S) - ceil_div(pos0, g.S);
       auto& pg = kv->pages[t];
       for (int k = 0; k < new_pages; ++k) {
-        const int32_t page = kv->free_stack.back();
-        kv->free_stack.pop_back();
+        const int32_t page = pop_page(kv);
         idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size();
         val[n_ids] = page;
         ++n_ids;
@@ -410,8 +446,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
     if (n_recs == 0) continue;
     // records hold absolute token indices; the kernel is launched over [tok_lo, tok_hi)
     for (int k = 0; k < n_recs; ++k) recs[k].tok0 -= tok_lo;
-    const size_t up_bytes = 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
-    // only the used prefixes of the three arrays need to travel
+    // only the used prefixes of the three arrays (records, table indices, page ids) need to travel
     if (cudaMemcpyAsync(slot->dev + 256, slot->host + 256, (size_t)n_recs * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
       return TIDE_ERR_CUDA;
     if (n_ids > 0) {
@@ -422,7 +457,14 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
         return TIDE_ERR_CUDA;
       ++kv->append_launches;
     }
-    (void)up_bytes;
+    if (n_cpy > 0) {
+      uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
+      if (cudaMemcpyAsync(dcpy, cpy_src, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (cudaMemcpyAsync(dcpy + (size_t)kSlotRecs * 4, cpy_dst, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (launch_copy_pages(kv->pool, (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), n_cpy, g.page_bytes, st) != cudaSuccess)
+        return TIDE_ERR_CUDA;
+      ++kv->append_launches;
+    }
     AppendParams ap;
     ap.pool = kv->pool;
     ap.table = kv->d_table;
@@ -451,6 +493,75 @@ int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k, void* 
   const int32_t* row = kv->d_table + (size_t)task * kv->g.max_pages_per_task;
   if (launch_read(kv->pool, row, 0, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
     return TIDE_ERR_CUDA;
+  return TIDE_OK;
+}
+
+int tide_kv_fork(tide_kv_t* kv, int32_t layer, int32_t parent, int32_t child, void* stream) {
+  if (kv == nullptr || layer != 0 || !task_in_range(kv, parent) || !task_in_range(kv, child)) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[parent]) return TIDE_ERR_UNKNOWN_TASK;
+  if (kv->live[child]) return TIDE_ERR_TASK_EXISTS;
+  const Geom& g = kv->g;
+  const int L = kv->len[parent];
+  const int n_full = L / g.S;
+  const bool partial = L % g.S != 0;
+  if (partial && kv->free_stack.empty()) return TIDE_ERR_NO_PAGES;
+  cudaStream_t st = (cudaStream_t)stream;
+  // ---- bookkeeping: share the full pages, take one fresh page for the copy of the partial one ----
+  auto& cp = kv->pages[child];
+  cp.assign(kv->pages[parent].begin(), kv->pages[parent].begin() + n_full);
+  for (int32_t page : cp) ++kv->refcnt[(size_t)page];
+  int32_t copy_src = -1, copy_dst = -1;
+  if (partial) {
+    copy_src = kv->pages[parent][(size_t)n_full];
+    copy_dst = pop_page(kv);
+    cp.push_back(copy_dst);
+  }
+  kv->live[child] = 1;
+  kv->len[child] = L;
+  kv->used_tokens += L;
+  // ---- device: the child's page-table row, then the page copy ----
+  for (size_t done = 0; done < cp.size();) {
+    Slot* slot;
+    int rc = acquire_slot(kv, &slot);
+    if (rc != TIDE_OK) return rc;
+    int32_t* idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
+    int32_t* val = idx + kSlotPageIds;
+    const size_t n = std::min(kSlotPageIds, cp.size() - done);
+    for (size_t i = 0; i < n; ++i) {
+      idx[i] = child * g.max_pages_per_task + (int32_t)(done + i);
+      val[i] = cp[done + i];
+    }
+    uint8_t* didx = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec);
+    if (cudaMemcpyAsync(didx, idx, n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaMemcpyAsync(didx + kSlotPageIds * 4, val, n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (launch_table_update(kv->d_table, (const int32_t*)didx, (const int32_t*)(didx + kSlotPageIds * 4), (int)n, st) != cudaSuccess)
+      return TIDE_ERR_CUDA;
+    done += n;
+    if (done == cp.size() && partial) {
+      int32_t* hc = val + kSlotPageIds;   // copy-pair area of the slot
+      hc[0] = copy_src;
+      hc[kSlotRecs] = copy_dst;
+      uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
+      if (cudaMemcpyAsync(dcpy, hc, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (cudaMemcpyAsync(dcpy + (size_t)kSlotRecs * 4, hc + kSlotRecs, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (launch_copy_pages(kv->pool, (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), 1, g.page_bytes, st) != cudaSuccess)
+        return TIDE_ERR_CUDA;
+    }
+    if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+  }
+  if (cp.empty() && partial) return TIDE_ERR_INVALID_ARG;   // unreachable: a partial page implies one entry
+  return TIDE_OK;
+}
+
+int tide_kv_page_refs(tide_kv_t* kv, int32_t task, int32_t* out, int32_t cap, int32_t* n_pages) {
+  if (kv == nullptr || n_pages == nullptr || !task_in_range(kv, task) || cap < 0) return TIDE_ERR_INVALID_ARG;
+  if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  const auto& pg = kv->pages[task];
+  *n_pages = (int32_t)pg.size();
+  if (out != nullptr) {
+    if ((size_t)cap < pg.size()) return TIDE_ERR_INVALID_ARG;
+    for (size_t i = 0; i < pg.size(); ++i) out[i] = kv->refcnt[(size_t)pg[i]];
+  }
   return TIDE_OK;
 }
 
@@ -692,7 +803,8 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
   uint8_t* dout = kv->ws + kv->lay.off_stage_out;
   float* dlse = (float*)(kv->ws + kv->lay.off_stage_lse);
   const size_t kv_bytes = T * g.Hkv * g.D * 2, q_bytes = T * g.Hq * g.D * 2;
-  // validate the append (duplicates, pages) BEFORE any copy by running it first: it is all-or-nothing
+  // The copies only fill the staging area; tide_kv_append then validates everything (duplicates, pages)
+  // before it changes any state, so a rejected step leaves the cache as it was.
   if (cudaMemcpyAsync(dk, new_k, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
   if (cudaMemcpyAsync(dv, new_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
   if (cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;

@@ -46,7 +46,7 @@ EXPORTS = [
     "tide_strerror", "tide_kv_required_bytes", "tide_kv_create", "tide_kv_destroy", "tide_kv_reset",
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
-    "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune",
+    "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune", "tide_kv_fork", "tide_kv_page_refs",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -157,6 +157,16 @@ class TideKV:
 
     def release(self, task):
         _check(lib.tide_kv_release(self.handle, ctypes.c_int32(task)), "tide_kv_release")
+
+    def fork(self, parent, child, stream=None):
+        _check(lib.tide_kv_fork(self.handle, ctypes.c_int32(0), ctypes.c_int32(parent), ctypes.c_int32(child), _stream(stream)), "tide_kv_fork")
+
+    def page_refs(self, task):
+        n = ctypes.c_int32(0)
+        _check(lib.tide_kv_page_refs(self.handle, ctypes.c_int32(task), None, ctypes.c_int32(0), ctypes.byref(n)), "tide_kv_page_refs")
+        out = np.empty(n.value, dtype=np.int32)
+        _check(lib.tide_kv_page_refs(self.handle, ctypes.c_int32(task), _ptr(out), ctypes.c_int32(n.value), ctypes.byref(n)), "tide_kv_page_refs")
+        return out
 
     def release_many(self, task_ids):
         ids = _i32(task_ids)

@@ -1,0 +1,129 @@
+"""Group-shared prefix pages on the GPU against the oracle (tide_kv_fork, reference-counted pages, the private
+copy an append takes before writing into a shared page).  A GRPO group rolls out G trajectories from one prompt
+(paper Section 2.1) and CTB keeps the group on the rank that holds its shared prefix (end of Section 4)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import cbuild
+from oracle.paged_kv import OracleError, PagedKVOracle
+from paper_2608_10402_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+HQ, HKV, D, S = 28, 4, 128, 16
+
+
+def _same(kv, orc, tasks):
+    for t in tasks:
+        assert kv.task_len(t) == orc.task_len(t)
+        assert np.array_equal(kv.page_table(t), orc.page_table(t)), f"page table of task {t}"
+        assert np.array_equal(kv.page_refs(t), orc.page_refs(t)), f"reference counts of task {t}"
+        gk, gv = kv.read(t)
+        ok, ov = orc.read(t)
+        assert np.array_equal(H.from_dev(gk), ok) and np.array_equal(H.from_dev(gv), ov), f"cache bits of task {t}"
+    assert kv.usage() == (orc.used_tokens(), orc.free_pages())
+
+
+def test_grpo_group_shares_its_prompt_pages():
+    import torch
+    from paper_2608_10402_b200 import tide
+    rng = np.random.default_rng(77)
+    P, G = 400, 8
+    order = rng.permutation(P).astype(np.int32)
+    kv = tide.TideKV(HQ, HKV, D, S, P, 16, 128, 16, 4096, free_order=order)
+    orc = PagedKVOracle(P, S, HKV, D, 16, 128, free_order=order)
+    scale = 1.0 / math.sqrt(D)
+    # the prompt is prefilled once ...
+    L0 = 1000 + 7                                            # ends inside a page: the partial page must be copied
+    pk_, pv_ = inputs.normal_bf16(rng, (L0, HKV, D)), inputs.normal_bf16(rng, (L0, HKV, D))
+    for o in (kv, orc):
+        o.alloc(0)
+    kv.append([0], [0, L0], H.to_dev(pk_, torch), H.to_dev(pv_, torch))
+    orc.append([0], [0, L0], pk_, pv_)
+    free_after_prompt = orc.free_pages()
+    # ... and the other G-1 trajectories fork from it
+    for c in range(1, G):
+        kv.fork(0, c)
+        orc.fork(0, c)
+    assert orc.free_pages() == free_after_prompt - (G - 1)   # one copied page per child, nothing else
+    _same(kv, orc, range(G))
+    # every trajectory continues on its own: a first action (decode), then an observation of its own length
+    for n_new in ([1] * G, [int(x) for x in rng.integers(20, 300, size=G)]):
+        indptr = np.concatenate([[0], np.cumsum(n_new)]).astype(np.int32)
+        T = int(indptr[-1])
+        nk, nv, q = (inputs.normal_bf16(rng, (T, HKV, D)), inputs.normal_bf16(rng, (T, HKV, D)),
+                     inputs.normal_bf16(rng, (T, HQ, D)))
+        kv.append(list(range(G)), indptr, H.to_dev(nk, torch), H.to_dev(nv, torch))
+        orc.append(list(range(G)), indptr, nk, nv)
+        rows = [(t, n_new[t], orc.task_len(t)) for t in range(G)]
+        out = torch.zeros((T, HQ, D), dtype=torch.int16, device="cuda")
+        lse = torch.zeros((T, HQ), dtype=torch.float32, device="cuda")
+        kv.attend(rows, H.to_dev(q, torch), scale, out, lse)
+        assert kv.status() == tide.OK
+        ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
+        H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, "group step")
+        _same(kv, orc, range(G))
+    # the prompt's pages survive until the last trajectory of the group is released
+    shared = set(int(p) for p in orc.page_table(0)[: L0 // S])
+    kv.release_many(list(range(G - 1)))
+    orc.release_many(list(range(G - 1)))
+    assert shared <= set(int(p) for p in orc.page_table(G - 1)) and not shared & set(orc.free)
+    _same(kv, orc, [G - 1])
+    kv.release(G - 1)
+    orc.release(G - 1)
+    assert kv.usage() == (0, P)
+    kv.close()
+
+
+def test_random_ops_with_forks_match_the_oracle_bit_for_bit():
+    import torch
+    from paper_2608_10402_b200 import tide
+    rng = np.random.default_rng(5)
+    P, NT = 96, 10
+    order = rng.permutation(P).astype(np.int32)
+    kv = tide.TideKV(8, 2, 64, 16, P, NT, 12, NT, 512, free_order=order)
+    orc = PagedKVOracle(P, 16, 2, 64, NT, 12, free_order=order)
+    codes = {"fork": 0, "append": 0, "truncate": 0, "release": 0, "errors": 0}
+    for step in range(250):
+        live = sorted(orc.live)
+        r = rng.random()
+        op = None
+        if r < 0.15 or not live:
+            t = int(rng.integers(0, NT))
+            op = ("alloc", lambda o, t=t: o.alloc(t))
+        elif r < 0.35:
+            a, b = int(rng.choice(live)), int(rng.integers(0, NT))
+            op = ("fork", lambda o, a=a, b=b: o.fork(a, b))
+        elif r < 0.7:
+            t, n = int(rng.choice(live)), int(rng.integers(0, 40))
+            nk, nv = inputs.normal_bf16(rng, (n, 2, 64)), inputs.normal_bf16(rng, (n, 2, 64))
+            op = ("append", lambda o, t=t, n=n, nk=nk, nv=nv: o.append([t], [0, n], *((H.to_dev(nk, torch), H.to_dev(nv, torch)) if o is kv else (nk, nv))))
+        elif r < 0.85:
+            t = int(rng.choice(live))
+            nl = int(rng.integers(0, orc.task_len(t) + 1))
+            op = ("truncate", lambda o, t=t, nl=nl: o.truncate(t, nl))
+        else:
+            t = int(rng.choice(live))
+            op = ("release", lambda o, t=t: o.release(t))
+        name, fn = op
+        want = None
+        try:
+            fn(orc)
+        except OracleError as e:
+            want = e.code
+        if want is None:
+            fn(kv)
+            codes[name] = codes.get(name, 0) + 1
+        else:
+            with pytest.raises(tide.TideError) as e:
+                fn(kv)
+            assert e.value.code == want, (name, e.value.code, want)
+            codes["errors"] += 1
+        if step % 10 == 9:
+            _same(kv, orc, sorted(orc.live))
+    _same(kv, orc, sorted(orc.live))
+    assert codes["fork"] > 5 and codes["errors"] > 3, codes
+    kv.close()

@@ -245,3 +245,106 @@ def test_prune_keeps_prefix_and_tail_and_reuses_pages():
     with pytest.raises(OracleError) as e:
         c.release_many([2, 2])
     assert e.value.code == pk.ERR_DUPLICATE_TASK and 2 in c.live
+
+
+def test_fork_shares_full_pages_and_copies_the_partial_one():
+    # hand trace, page size 4, pool of 8 handed out in order 0..7
+    c = PagedKVOracle(8, 4, 1, 2, 4, 6)
+    k = np.arange(40 * 2, dtype=np.uint16).reshape(40, 1, 2)
+    v = k + np.uint16(1000)
+    c.alloc(0)
+    c.append([0], [0, 10], k[:10], v[:10])                 # pages [0,1,2], the last one partial (2 of 4 slots)
+    c.fork(0, 1)                                           # child: shares 0,1; page 3 is a copy of page 2
+    assert list(c.page_table(1)) == [0, 1, 3] and list(c.page_refs(1)) == [2, 2, 1]
+    assert list(c.page_refs(0)) == [2, 2, 1] and c.free_pages() == 4
+    assert np.array_equal(c.read(1)[0], k[:10]) and np.array_equal(c.read(1)[1], v[:10])
+    # the two diverge: each appends into its own partial page, then takes fresh pages
+    c.append([0, 1], [0, 3, 9], k[10:19], v[10:19])         # parent +3 (fills page 2, pops 4), child +6 (fills 3, pops 5)
+    assert list(c.page_table(0)) == [0, 1, 2, 4] and list(c.page_table(1)) == [0, 1, 3, 5]
+    assert np.array_equal(c.read(0)[0], np.concatenate([k[:10], k[10:13]]))
+    assert np.array_equal(c.read(1)[0], np.concatenate([k[:10], k[13:19]]))
+    # fork on a page boundary copies nothing
+    c.truncate(1, 8)
+    assert list(c.page_table(1)) == [0, 1] and c.free_stack_top_first()[:2] == [3, 5]
+    c.fork(1, 2)
+    assert list(c.page_table(2)) == [0, 1] and list(c.page_refs(2)) == [3, 3] and c.free_pages() == 4
+    # releasing the parent keeps the shared pages alive; the last holder frees them, last page first
+    c.release(0)
+    assert c.free_stack_top_first()[:2] == [2, 4] and list(c.page_refs(1)) == [2, 2]
+    c.release(1)
+    c.release(2)
+    assert c.free_pages() == 8 and c.free_stack_top_first()[:2] == [0, 1] and not c.ref
+
+
+def test_append_into_a_shared_partial_page_takes_a_private_copy_first():
+    c = PagedKVOracle(8, 4, 1, 2, 4, 6)
+    k = np.arange(40 * 2, dtype=np.uint16).reshape(40, 1, 2)
+    c.alloc(0)
+    c.append([0], [0, 8], k[:8], k[:8])                    # pages [0,1], both full
+    c.fork(0, 1)                                           # child shares both
+    c.truncate(1, 6)                                       # child now ends INSIDE shared page 1
+    assert list(c.page_table(1)) == [0, 1] and c.ref[1] == 2
+    c.append([1], [0, 3], k[20:23], k[20:23])              # private copy of page 1 (pops 2), then one more page (3)
+    assert list(c.page_table(1)) == [0, 2, 3] and c.ref[1] == 1 and c.ref[2] == 1
+    assert np.array_equal(c.read(1)[0], np.concatenate([k[:6], k[20:23]]))
+    assert np.array_equal(c.read(0)[0], k[:8])             # the parent still sees its own tokens 6 and 7
+    # the extra page counts in the all-or-nothing check: 4 pages free, child 2 needs a copy + 4 new pages
+    c.fork(0, 2)
+    c.truncate(2, 5)
+    before = c.state_hash()
+    with pytest.raises(OracleError) as e:
+        c.append([2], [0, 16], k[:16], k[:16])             # ceil(21/4) - 2 = 4 new pages + 1 copy = 5 > 4 free
+    assert e.value.code == pk.ERR_NO_PAGES and c.state_hash() == before
+    with pytest.raises(OracleError) as e:
+        c.fork(0, 1)
+    assert e.value.code == pk.ERR_TASK_EXISTS
+
+
+def test_refcount_conservation_under_random_ops_with_forks():
+    rng = np.random.default_rng(31)
+    P, S = 48, 4
+    c = PagedKVOracle(P, S, 1, 2, max_tasks=10, max_pages_per_task=12, free_order=rng.permutation(P))
+    shadow = {}
+    counter = 0
+    for _ in range(600):
+        r = rng.random()
+        live = sorted(c.live)
+        try:
+            if r < 0.15:
+                t = int(rng.integers(0, 10))
+                c.alloc(t)
+                shadow[t] = []
+            elif r < 0.3 and live:
+                a, b = int(rng.choice(live)), int(rng.integers(0, 10))
+                c.fork(a, b)
+                shadow[b] = list(shadow[a])
+            elif r < 0.7 and live:
+                t = int(rng.choice(live))
+                n = int(rng.integers(0, 9))
+                kk = (np.arange(n * 2, dtype=np.uint32) + counter).astype(np.uint16).reshape(n, 1, 2)
+                counter += 2 * n
+                c.append([t], [0, n], kk, kk ^ np.uint16(0xAAAA))
+                shadow[t].extend(kk[i].copy() for i in range(n))
+            elif r < 0.85 and live:
+                t = int(rng.choice(live))
+                nl = int(rng.integers(0, c.task_len(t) + 1))
+                c.truncate(t, nl)
+                shadow[t] = shadow[t][:nl]
+            elif live:
+                t = int(rng.choice(live))
+                c.release(t)
+                del shadow[t]
+        except OracleError:
+            pass
+        held = {}
+        for t in c.live:
+            assert len(c.pages[t]) == -(-c.len[t] // S)
+            for p in c.pages[t]:
+                held[p] = held.get(p, 0) + 1
+        assert held == c.ref, "reference counts disagree with the page tables"
+        assert not set(held) & set(c.free) and len(held) + c.free_pages() == P
+    for t in c.live:
+        kk, _ = c.read(t)
+        assert kk.shape[0] == len(shadow[t])
+        for pos, row in enumerate(shadow[t]):
+            assert np.array_equal(kk[pos], row)
