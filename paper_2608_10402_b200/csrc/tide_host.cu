@@ -74,7 +74,8 @@ struct tide_kv {
   cudaEvent_t ev_append[2] = {nullptr, nullptr};
   cudaEvent_t ev_attend[4] = {nullptr, nullptr, nullptr, nullptr};
   bool have_append_times = false, have_attend_times = false;
-  int umma_min_rows = kUmmaTileRows;  // packed rows from which a resume row takes the tcgen05 path
+  int umma_min_rows = kDecodeTileRows + 1;  // packed rows from which a resume row takes the tcgen05 path (measured:
+                                            // it beats the warp-MMA tile path from the first row beyond a decode item)
   int items_per_sm = kTargetItemsPerSm;  // work items the planner aims for per SM
 };
 
