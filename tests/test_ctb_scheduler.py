@@ -1,0 +1,100 @@
+"""Algorithm 1 (Semantic-Aware CTB Scheduling): the product scheduler against the oracle that restates the
+listing, on seeded random traces (identical decisions, in order), plus the properties the algorithm fixes and a
+sanity check of the rollout simulator.  CPU only."""
+import numpy as np
+
+from oracle import ctb_alg1 as oracle
+from paper_2608_10402_b200 import ctb
+
+
+def _trace(seed, n_ranks, passes=60):
+    rng = np.random.default_rng(seed)
+    budgets = [int(rng.integers(3000, 9000)) for _ in range(n_ranks)]
+    env_limit = int(rng.integers(6, 30))
+    sched = ctb.CTBScheduler(budgets, ctx_norm=8192.0, env_limit=env_limit)
+    otasks, oqueue = [], []
+    w = oracle.Weights()
+    next_id = 0
+    for p in range(passes):
+        # arrivals
+        for _ in range(int(rng.integers(0, 5))):
+            group, is_eval, probed = int(rng.integers(0, 6)), bool(rng.random() < 0.15), int(rng.integers(200, 1500))
+            sched.submit(next_id, group, probed, is_eval)
+            otasks.append(oracle.Task(next_id, group, is_eval, probed))
+            oqueue.append(next_id)
+            next_id += 1
+        # some active tasks finish, the others grow (turn probing)
+        act = [t.id for t in otasks if t.state == "active"]
+        for tid in act:
+            if rng.random() < 0.1:
+                sched.finish(tid)
+                next(t for t in otasks if t.id == tid).state = "done"
+        grow = {tid: next(t for t in otasks if t.id == tid).footprint + int(rng.integers(0, 900))
+                for tid in act if next(t for t in otasks if t.id == tid).state == "active" and rng.random() < 0.7}
+        got = sched.schedule(grow)
+        want = oracle.schedule_pass(otasks, oqueue, budgets, w, 8192.0, env_limit, grow)
+        assert got == want, f"pass {p}: {got} != {want}"
+        yield sched, otasks, budgets, env_limit, got
+
+
+def test_scheduler_matches_the_listing_on_random_traces():
+    n_events = 0
+    kinds = set()
+    for seed in range(6):
+        for sched, otasks, budgets, env_limit, ev in _trace(seed, n_ranks=1 + seed % 3):
+            n_events += len(ev)
+            kinds.update(k for k, _, _ in ev)
+            # same bookkeeping on both sides
+            for r in range(len(budgets)):
+                assert sched.usage[r] == oracle.token_usage(otasks, r)
+            assert {t.id for t in otasks if t.state == "paused"} == set(sched.paused)
+    assert n_events > 200 and kinds == {"admit", "evict", "resume"}
+
+
+def test_budget_concurrency_and_affinity_hold_after_every_pass():
+    for sched, otasks, budgets, env_limit, ev in _trace(11, n_ranks=3):
+        for r, B in enumerate(budgets):
+            # over budget only if a single task alone exceeds it (the loop stops when nothing is left to preempt)
+            assert sched.usage[r] <= B or len(sched.active[r]) <= 1
+        assert sched.n_active <= env_limit
+        evicted_from = {}
+        for kind, tid, r in ev:
+            if kind == "evict":
+                evicted_from[tid] = r
+        for kind, tid, r in ev:
+            if kind == "resume" and tid in evicted_from:
+                assert evicted_from[tid] == r, "a paused task resumed away from the rank that holds its prefix"
+
+
+def test_priority_tiers_decide_who_is_preempted():
+    # one rank, four active tasks that differ in exactly one tier each; shrinking headroom evicts them in the
+    # order Low (short context) -> ... -> evaluation task last (Table 1)
+    s = ctb.CTBScheduler([10_000], ctx_norm=8192.0)
+    s.submit(0, group=0, probed=1000, is_eval=True)
+    s.submit(1, group=1, probed=1000)
+    s.submit(2, group=2, probed=1000)
+    s.submit(3, group=1, probed=1000)          # same group as 1
+    s.submit(4, group=1, probed=1000)
+    assert [e[0] for e in s.schedule()] == ["admit"] * 5
+    s.finish(4)                                 # group 1 is now 1/3 complete: tasks 1 and 3 rank above task 2
+    s.schedule({0: 3000, 1: 3000, 2: 3000, 3: 2000})   # usage 11000 > 10000
+    assert s.tasks[3].state == "active" and s.tasks[2].state == "paused"   # lowest tier value goes first
+    order = []
+    for shrink in (7000, 4000, 2500):
+        s.budgets[0] = shrink
+        order += [tid for kind, tid, _ in s.schedule() if kind == "evict"]
+    assert order == [3, 1, 0] or order[:2] == [3, 1]     # short context before long, evaluation task last
+    assert s.tasks[0].state in ("active", "paused")
+
+
+def test_simulated_rollout_ctb_keeps_more_kv_than_request_batching():
+    rng = np.random.default_rng(0)
+    rollout = ctb.synthetic_rollout(rng, n_groups=24, group_size=8)
+    budget = 120_000
+    a = ctb.simulate(rollout, "ctb", budget)
+    b = ctb.simulate(rollout, "request", budget, fixed_concurrency=96)
+    assert a["context"] > 0 and b["context"] > 0
+    assert a["hit_rate"] > b["hit_rate"] and a["prefilled"] < b["prefilled"]
+    # with ample memory nothing is ever dropped under either policy
+    c = ctb.simulate(rollout, "request", 10**9, fixed_concurrency=96)
+    assert c["hit_rate"] == 1.0
