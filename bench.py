@@ -122,6 +122,94 @@ def build_state(w, torch, tide, seed):
     return kv, new_k, new_v, q, out, lse
 
 
+def multi_layer_leg(args, w, torch, tide, seed):
+    """The same step over `--layers` K/V stores (one per model layer) that share one page table: device time per
+    layer when every layer is driven by its own write + attend calls (the work is planned once per layer), when
+    the step is planned once (tide_step_begin) and every layer only launches kernels (tide_step_layer), and when
+    those launches are replayed from a CUDA graph captured for this step."""
+    L = args.layers
+    total_q = int(w.n_new.sum())
+    kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task, max_batch_rows=w.B,
+                     max_batch_tokens=total_q, free_order=w.free_order, num_layers=L)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    for b in range(w.B):
+        kv.alloc(int(w.task[b]))
+    for b in range(w.B):
+        p = int(w.prefix[b])
+        k = torch.randn((p, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+        v = torch.randn((p, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+        kv.extend([int(w.task[b])], [0, p])
+        for l in range(L):
+            kv.write(l, [int(w.task[b])], [0, p], k, v)
+    new_k = torch.randn((L, total_q, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+    new_v = torch.randn((L, total_q, w.Hkv, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+    q = torch.randn((L, total_q, w.Hq, w.D), device="cuda", generator=gen).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    lse = torch.empty((L, total_q, w.Hq), device="cuda", dtype=torch.float32)
+    rows = tide.rows_array(w.rows())
+    ids = np.asarray(w.task, dtype=np.int32)
+    indptr = np.concatenate([[0], np.cumsum(w.n_new)]).astype(np.int32)
+    order_back = [(int(w.task[b]), int(w.prefix[b])) for b in reversed(range(w.B))]
+    stream = torch.cuda.Stream()
+
+    def rollback():
+        for t, p in order_back:
+            kv.truncate(t, p)
+
+    def per_layer_calls():
+        kv.extend(ids, indptr, stream=stream)
+        for l in range(L):
+            kv.write(l, ids, indptr, new_k[l], new_v[l], stream=stream)
+            kv.attend(rows, q[l], w.scale, out[l], lse[l], layer=l, stream=stream)
+
+    def planned():
+        kv.step_begin(rows, stream=stream)
+        for l in range(L):
+            kv.step_layer(l, new_k[l], new_v[l], q[l], w.scale, out[l], lse[l], stream=stream)
+
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        kv.step_begin(rows, stream=stream)
+        t0 = time.perf_counter()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for l in range(L):
+                kv.step_layer(l, new_k[l], new_v[l], q[l], w.scale, out[l], lse[l], stream=torch.cuda.current_stream())
+        capture_ms = (time.perf_counter() - t0) * 1e3
+        rollback()
+
+        def from_graph():
+            kv.step_begin(rows, stream=stream)      # the same rows give the same plan at the same place
+            graph.replay()
+
+        res = {}
+        for name, fn in (("per_layer_calls", per_layer_calls), ("planned", planned), ("graph", from_graph)):
+            for _ in range(3):
+                fn()
+                rollback()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                fn()
+                rollback()
+            e1.record(stream)
+            stream.synchronize()
+            host = []
+            for _ in range(args.steps):          # host time to enqueue one step on an idle stream
+                t0 = time.perf_counter()
+                fn()
+                host.append((time.perf_counter() - t0) * 1e3)
+                rollback()
+                stream.synchronize()
+            res[name] = {"device_ms_per_layer": e0.elapsed_time(e1) / args.steps / L,
+                         "host_enqueue_ms_per_step": float(np.median(host))}
+        assert kv.status(stream=stream) == tide.OK
+    kv.close()
+    return {"layers": L, "graph_capture_ms": capture_ms, **res}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -219,6 +307,14 @@ def run_ours(args):
     kv_gbs = replicas.whole_job_rate(dec_bytes_all, dec_ms) / 1e9
     tflops = replicas.whole_job_rate(res_flops_all, tile_ms) / 1e12
 
+    multi_layer = None
+    if args.layers > 1:
+        kv.close()
+        kv.pool = kv.workspace = None
+        del new_k, new_v, q, out, lse
+        torch.cuda.empty_cache()
+        multi_layer = multi_layer_leg(args, w, torch, tide, seed=rank)
+
     if rank == 0:
         reduced = args.tasks is not None or args.len_div != 1 or args.pool_factor is not None
         n_app = int(w.n_new.sum())
@@ -262,6 +358,8 @@ def run_ours(args):
             "gpu_launches": int(launches_per_step * args.steps),
             "clocks": clocks,
         }
+        if multi_layer is not None:
+            line["multi_layer"] = multi_layer
         line["cpu_baseline"] = cpu_baseline(args.config, budget_s=args.cpu_budget)
         print(json.dumps(line))
     kv.close()
@@ -352,6 +450,8 @@ def main():
     ap.add_argument("--tasks", type=int, default=None, help="fewer tasks (profiler captures only)")
     ap.add_argument("--len-div", type=int, default=1, help="divide every length bound (profiler captures only)")
     ap.add_argument("--pool-factor", type=float, default=None, help="pool pages / live pages (profiler captures only)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="> 1 adds a leg that steps this many layers over one page table (planned once, CUDA graph)")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -62,7 +62,8 @@ typedef struct {
 } tide_row_t;
 
 typedef struct {
-  int32_t num_layers;         /* must be 1                                                          */
+  int32_t num_layers;         /* L in [1, 256]: K/V stores that share one page table (layer l of a   */
+                              /* model); the pool holds L * num_pages pages                         */
   int32_t num_q_heads;        /* Hq, a multiple of num_kv_heads, Hq/Hkv <= 16                       */
   int32_t num_kv_heads;       /* Hkv                                                                */
   int32_t head_dim;           /* D: 64 or 128                                                       */
@@ -108,6 +109,20 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
                    const int32_t* indptr /*host, n_tasks+1*/, const void* new_k /*device*/,
                    const void* new_v /*device*/, void* stream);
 
+/* A model with L layers keeps L K/V stores that grow in lock step: one page table and one set of lengths serve
+ * all of them (the paper's token budget of Section 4.1 counts tokens, not layers).  With num_layers > 1 an
+ * append is therefore split: tide_kv_extend grows the tasks once per step (pages, lengths, the device page
+ * table, and on every layer the private copy of a shared partial page) and writes no K/V;
+ * tide_kv_write(layer) then puts that layer's new rows into the LAST indptr[j+1]-indptr[j] positions of
+ * task_ids[j] (TIDE_ERR_CTX_RANGE if a task is shorter than that).  tide_kv_append is tide_kv_extend followed by
+ * tide_kv_write on layer 0, and accepts layer 0 only.  Argument meaning, all-or-nothing behaviour and errors
+ * are those of tide_kv_append. */
+int tide_kv_extend(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids /*host*/,
+                   const int32_t* indptr /*host, n_tasks+1*/, void* stream);
+int tide_kv_write(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids /*host*/,
+                  const int32_t* indptr /*host, n_tasks+1*/, const void* new_k /*device*/,
+                  const void* new_v /*device*/, void* stream);
+
 /* Attention of a mixed continuous batch over the cache (Section 3.2: concurrent multi-task
  * generation on one rank; Section 4: resumed tasks continue from preserved state).
  * Row b: query i in [0, q_len) sits at position ctx_len - q_len + i and sees keys [0, that position]
@@ -129,6 +144,20 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
                    const void* new_k /*host*/, const void* new_v /*host*/, const void* q /*host*/,
                    float scale, void* out /*host*/, float* lse /*host or NULL*/, void* stream);
 
+/* One CTB step of a model with several layers, planned once.  tide_step_begin takes the step's rows (distinct
+ * tasks; ctx_len must equal the resident length after q_len tokens are added, as in tide_step_host), grows the
+ * tasks (tide_kv_extend), plans the attention work and uploads the plan and the write records to a part of the
+ * workspace that stays valid until the next tide_step_begin or any call that changes a task.  All-or-nothing.
+ * tide_step_layer(layer) then writes that layer's new_k / new_v (device bf16 [sum q_len, Hkv, D], batch order)
+ * and attends q against layer `layer` exactly as tide_attend would; it only launches kernels (no copies, no
+ * events, no host waits), so the calls of all layers may be captured in one CUDA graph and replayed, as long
+ * as the captured pointers stay valid.  scale must be positive and finite.  TIDE_ERR_INVALID_ARG if no step is
+ * open.  Per-phase timing (tide_set_profiling) does not cover tide_step_layer. */
+int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows /*host*/, void* stream);
+int tide_step_layer(tide_kv_t* kv, int32_t layer, const void* new_k /*device*/, const void* new_v /*device*/,
+                    const void* q /*device*/, float scale, void* out /*device*/, float* lse /*device or NULL*/,
+                    void* stream);
+
 /* Return the task's pages to the free stack, last page first, and forget the task (task end or
  * eviction, Algorithm 1).  Host only; page contents are not cleared. */
 int tide_kv_release(tide_kv_t* kv, int32_t task);
@@ -143,8 +172,9 @@ int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len);
  * never written again), a partial last page is copied into a fresh page, so parent and child can both keep
  * appending.  A page returns to the free stack when its last holder lets go of it.  An append that would write
  * into a page other tasks still hold (possible after tide_kv_truncate into shared pages) first replaces it by
- * a private copy, taken from the free stack before the task's other new pages.  Errors: TIDE_ERR_TASK_EXISTS,
- * TIDE_ERR_UNKNOWN_TASK, TIDE_ERR_NO_PAGES (no page for the copy). */
+ * a private copy, taken from the free stack before the task's other new pages.  Page copies cover every
+ * layer; `layer` must be 0.  Errors: TIDE_ERR_TASK_EXISTS, TIDE_ERR_UNKNOWN_TASK, TIDE_ERR_NO_PAGES (no page
+ * for the copy). */
 int tide_kv_fork(tide_kv_t* kv, int32_t layer, int32_t parent, int32_t child, void* stream);
 /* How many tasks hold each page of `task` (same order as tide_kv_page_table). */
 int tide_kv_page_refs(tide_kv_t* kv, int32_t task, int32_t* out /*host*/, int32_t cap, int32_t* n_pages);
@@ -157,7 +187,11 @@ int tide_kv_release_many(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids
  * the trajectory): the task keeps tokens [0, keep_prefix) and [tail_begin, len); the tokens in between are
  * dropped and the tail moves down to start at keep_prefix.  Equivalent, page table included, to reading the
  * tail, tide_kv_truncate(task, keep_prefix) and appending the tail again; the move runs on `stream` through
- * the workspace staging area.  Requires 0 <= keep_prefix <= tail_begin <= len. */
+ * the workspace staging area and covers every layer (`layer` must be 0).  Requires
+ * 0 <= keep_prefix <= tail_begin <= len.  All-or-nothing: TIDE_ERR_NO_PAGES if the shorter task could not get
+ * its pages (only possible when it shares pages, which do not come back to the free stack);
+ * TIDE_ERR_WORKSPACE if the task shares a page from position keep_prefix on and its tail is longer than
+ * max_batch_tokens (such a tail has to be staged whole). */
 int tide_kv_prune(tide_kv_t* kv, int32_t layer, int32_t task, int32_t keep_prefix, int32_t tail_begin, void* stream);
 
 /* Introspection (the per-rank token usage CTB schedules on, Section 4.1 / Algorithm 1). */

@@ -265,11 +265,19 @@ class PagedKVOracle:
             k, v = self.read(task)
             tail_k, tail_v = k[tail_begin:].copy(), v[tail_begin:].copy()
         n_tail = self.len[task] - tail_begin
+        # like every call, prune changes nothing when it has to refuse: remember the bookkeeping, and put it
+        # back if the append of the tail finds too few pages (possible only when the task shares pages, since
+        # shared pages do not return to the free stack when the task lets go of them)
+        before = (list(self.free), dict(self.len), {t: list(p) for t, p in self.pages.items()}, dict(self.ref))
         self.truncate(task, keep_prefix)
-        if self.store_values:
-            self.append([task], [0, n_tail], tail_k, tail_v)
-        else:
-            self.append([task], [0, n_tail])
+        try:
+            if self.store_values:
+                self.append([task], [0, n_tail], tail_k, tail_v)
+            else:
+                self.append([task], [0, n_tail])
+        except OracleError:
+            self.free, self.len, self.pages, self.ref = before
+            raise
 
     def reset(self, free_order=None):
         """Flush every task (the cache flush at a weight synchronisation,

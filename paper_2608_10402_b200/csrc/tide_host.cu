@@ -28,10 +28,26 @@ constexpr long long kPartRowsBase = 256 * 1024;
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t off_status, off_table, off_meta, off_part_o, off_part_lse, off_stage_k, off_stage_v, off_stage_q,
-      off_stage_out, off_stage_lse, total;
+  size_t off_status, off_table, off_old_row, off_step, off_meta, off_part_o, off_part_lse, off_stage_k, off_stage_v,
+      off_stage_q, off_stage_out, off_stage_lse, total;
   size_t slot_bytes;
+  size_t step_bytes;      // held plan of a multi-layer step: write records, then segments
+  size_t step_seg_off;    // offset of the segments inside the step area
   long long part_rows;
+};
+
+// A planned batch as the launches need it: where the four segment arrays sit on the device and how many work
+// items each launch has.
+struct PlanDev {
+  const Segment* segs = nullptr;   // [decode][tile][tcgen05][merge]
+  size_t n_dec = 0, n_tile = 0, n_umma = 0, n_merge = 0;
+  long long items_dec = 0, items_tile = 0, items_umma = 0, merge_rows = 0;
+};
+
+struct PlanHost {
+  std::vector<Segment> seg_dec, seg_tile, seg_umma, seg_merge;
+  long long items_dec = 0, items_tile = 0, items_umma = 0, merge_rows = 0;
+  size_t n_all() const { return seg_dec.size() + seg_tile.size() + seg_umma.size() + seg_merge.size(); }
 };
 
 struct Slot {
@@ -49,8 +65,10 @@ struct tide_kv {
   Layout lay;
   int device = 0;
   uint8_t* pool = nullptr;
+  size_t layer_stride = 0;  // bytes between the page pools of consecutive layers
   uint8_t* ws = nullptr;
   int32_t* d_table = nullptr;
+  int32_t* d_old_row = nullptr;  // one page-table row: what a task's row was before a prune changed it
   int* d_status = nullptr;
   float* d_part_o = nullptr;
   float* d_part_lse = nullptr;
@@ -77,13 +95,20 @@ struct tide_kv {
   int umma_min_rows = kDecodeTileRows + 1;  // packed rows from which a resume row takes the tcgen05 path (measured:
                                             // it beats the warp-MMA tile path from the first row beyond a decode item)
   int items_per_sm = kTargetItemsPerSm;  // work items the planner aims for per SM
+  // multi-layer step held between tide_step_begin and the tide_step_layer calls
+  uint8_t* h_step = nullptr;   // pinned staging of the step area
+  cudaEvent_t ev_step = nullptr;
+  bool step_upload_pending = false, step_valid = false;
+  PlanDev step_plan;
+  int step_recs = 0, step_tokens = 0;
+  uint8_t* layer_pool(int layer) const { return pool + (size_t)layer * layer_stride; }
 };
 
 namespace {
 
 bool valid_geometry(const tide_kv_config_t* c) {
   if (c == nullptr) return false;
-  if (c->num_layers != 1) return false;
+  if (c->num_layers < 1 || c->num_layers > 256) return false;
   if (c->num_kv_heads <= 0 || c->num_q_heads <= 0 || c->num_q_heads % c->num_kv_heads != 0) return false;
   if (c->num_q_heads / c->num_kv_heads > 16) return false;
   if (c->head_dim != 64 && c->head_dim != 128) return false;
@@ -110,6 +135,10 @@ Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
   size_t off = 0;
   L.off_status = off; off += 256;
   L.off_table = off; off = align_up(off + (size_t)c->max_tasks * c->max_pages_per_task * 4, 256);
+  L.off_old_row = off; off = align_up(off + (size_t)c->max_pages_per_task * 4 + 64, 256);   // row + one page pair
+  L.step_seg_off = align_up((size_t)c->max_batch_rows * sizeof(AppendRec), 256);
+  L.step_bytes = align_up(L.step_seg_off + (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
+  L.off_step = off; off += L.step_bytes;
   L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 + (size_t)kSlotRecs * 8 +
                               (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
   L.off_meta = off; off += L.slot_bytes * kSlots;
@@ -202,7 +231,7 @@ const char* tide_strerror(int code) {
 int tide_kv_required_bytes(const tide_kv_config_t* cfg, size_t* pool_bytes, size_t* workspace_bytes) {
   if (!valid_geometry(cfg)) return TIDE_ERR_INVALID_ARG;
   const Geom g = make_geom(cfg);
-  if (pool_bytes) *pool_bytes = (size_t)cfg->num_pages * (size_t)g.page_bytes;
+  if (pool_bytes) *pool_bytes = (size_t)cfg->num_layers * (size_t)cfg->num_pages * (size_t)g.page_bytes;
   if (workspace_bytes) *workspace_bytes = make_layout(cfg, g).total;
   return TIDE_OK;
 }
@@ -213,7 +242,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   if (((uintptr_t)cfg->pool & 1023) || ((uintptr_t)cfg->workspace & 255)) return TIDE_ERR_INVALID_ARG;
   const Geom g = make_geom(cfg);
   const Layout lay = make_layout(cfg, g);
-  if (cfg->pool_bytes < (size_t)cfg->num_pages * (size_t)g.page_bytes || cfg->workspace_bytes < lay.total)
+  if (cfg->pool_bytes < (size_t)cfg->num_layers * (size_t)cfg->num_pages * (size_t)g.page_bytes || cfg->workspace_bytes < lay.total)
     return TIDE_ERR_WORKSPACE;
   std::vector<uint8_t> seen;
   if (cfg->free_order && !is_permutation(cfg->free_order, cfg->num_pages, seen)) return TIDE_ERR_INVALID_ARG;
@@ -225,15 +254,19 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->g = g;
   kv->lay = lay;
   kv->pool = (uint8_t*)cfg->pool;
+  kv->layer_stride = (size_t)cfg->num_pages * (size_t)g.page_bytes;
   kv->ws = (uint8_t*)cfg->workspace;
   kv->d_status = (int*)(kv->ws + lay.off_status);
   kv->d_table = (int32_t*)(kv->ws + lay.off_table);
+  kv->d_old_row = (int32_t*)(kv->ws + lay.off_old_row);
   kv->d_part_o = (float*)(kv->ws + lay.off_part_o);
   kv->d_part_lse = (float*)(kv->ws + lay.off_part_lse);
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
   ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
+  ok = ok && cudaHostAlloc((void**)&kv->h_step, lay.step_bytes, cudaHostAllocDefault) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&kv->ev_step, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; ok && i < kSlots; ++i) {
     ok = cudaHostAlloc((void**)&kv->slots[i].host, lay.slot_bytes, cudaHostAllocDefault) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&kv->slots[i].ev, cudaEventDisableTiming) == cudaSuccess;
@@ -263,6 +296,8 @@ int tide_kv_destroy(tide_kv_t* kv) {
     if (kv->slots[i].ev) cudaEventDestroy(kv->slots[i].ev);
   }
   if (kv->h_status) cudaFreeHost(kv->h_status);
+  if (kv->h_step) cudaFreeHost(kv->h_step);
+  if (kv->ev_step) cudaEventDestroy(kv->ev_step);
   for (cudaEvent_t e : kv->ev_append) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : kv->ev_attend) if (e) cudaEventDestroy(e);
   delete kv;
@@ -278,6 +313,7 @@ int tide_kv_reset(tide_kv_t* kv, const int32_t* free_order) {
   for (auto& p : kv->pages) p.clear();
   std::fill(kv->refcnt.begin(), kv->refcnt.end(), 0);
   kv->used_tokens = 0;
+  kv->step_valid = false;
   prime_free_stack(kv, free_order);
   return TIDE_OK;
 }
@@ -295,6 +331,7 @@ int tide_kv_alloc(tide_kv_t* kv, int32_t task, int64_t reserve_tokens) {
 int tide_kv_release(tide_kv_t* kv, int32_t task) {
   if (kv == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
   if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
+  kv->step_valid = false;
   auto& pg = kv->pages[task];
   for (size_t i = pg.size(); i-- > 0;) unref_page(kv, pg[i]);
   pg.clear();
@@ -308,6 +345,7 @@ int tide_kv_truncate(tide_kv_t* kv, int32_t task, int32_t new_len) {
   if (kv == nullptr || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
   if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
   if (new_len < 0 || new_len > kv->len[task]) return TIDE_ERR_INVALID_ARG;
+  kv->step_valid = false;
   auto& pg = kv->pages[task];
   const size_t keep = (size_t)ceil_div(new_len, kv->g.S);
   while (pg.size() > keep) {
@@ -345,12 +383,9 @@ int tide_kv_usage(tide_kv_t* kv, int64_t* used_tokens, int64_t* free_pages) {
   return TIDE_OK;
 }
 
-int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr,
-                   const void* new_k, const void* new_v, void* stream) {
-  if (kv == nullptr || layer != 0 || n_tasks < 0) return TIDE_ERR_INVALID_ARG;
-  if (n_tasks == 0) return TIDE_OK;
+// Range, liveness and duplicate checks shared by every call that takes a (task_ids, indptr) list.
+static int check_task_list(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr) {
   if (task_ids == nullptr || indptr == nullptr || indptr[0] != 0) return TIDE_ERR_INVALID_ARG;
-  const Geom& g = kv->g;
   for (int j = 0; j < n_tasks; ++j)
     if (indptr[j + 1] < indptr[j]) return TIDE_ERR_INVALID_ARG;
   for (int j = 0; j < n_tasks; ++j) {
@@ -365,9 +400,17 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
     if (kv->mark[task_ids[j]] == kv->mark_gen) return TIDE_ERR_DUPLICATE_TASK;
     kv->mark[task_ids[j]] = kv->mark_gen;
   }
-  const int T = indptr[n_tasks];
-  if (T > 0 && (new_k == nullptr || new_v == nullptr || ((uintptr_t)new_k & 15) || ((uintptr_t)new_v & 15)))
-    return TIDE_ERR_INVALID_ARG;
+  return TIDE_OK;
+}
+
+// Grows task_ids[j] by indptr[j+1]-indptr[j] tokens: host tables first, then the device page table, in uploads of
+// bounded size.  No K/V is written.  A task that ends inside a page that other tasks hold gets a private copy of
+// that page before its other pages are taken: with cow_out == nullptr the copy runs here on every layer, otherwise
+// the (old, new) page pairs are handed back and the caller copies (it may have to read the old pages first).
+// The task list must have passed check_task_list.
+static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, cudaStream_t st,
+                        std::vector<int32_t>* cow_out) {
+  const Geom& g = kv->g;
   long long need = 0;
   for (int j = 0; j < n_tasks; ++j) {
     const int t = task_ids[j], c = indptr[j + 1] - indptr[j];
@@ -379,77 +422,24 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
   }
   if (need > (long long)kv->free_stack.size()) return TIDE_ERR_NO_PAGES;
 
-  // ---- mutation: host tables first, then upload the deltas and scatter, in bounded batches ----
-  cudaStream_t st = (cudaStream_t)stream;
-  kv->append_launches = 0;
-  if (kv->profiling) cudaEventRecord(kv->ev_append[0], st);
-  int j = 0, done_in_task = 0;  // progress cursor: task index, tokens of that task already recorded
+  // ---- mutation ----
+  kv->step_valid = false;
+  Slot* slot = nullptr;
+  int32_t *idx = nullptr, *val = nullptr, *cpy_src = nullptr, *cpy_dst = nullptr;
+  size_t n_ids = 0;
+  int n_cpy = 0;
   int rc = TIDE_OK;
-  while (j < n_tasks) {
-    Slot* slot;
+  auto open_slot = [&]() -> int {
+    if (slot != nullptr) return TIDE_OK;
     if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
-    AppendRec* recs = (AppendRec*)(slot->host + 256);
-    int32_t* idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
-    int32_t* val = idx + kSlotPageIds;
-    int32_t* cpy_src = val + kSlotPageIds;
-    int32_t* cpy_dst = cpy_src + kSlotRecs;
-    int n_recs = 0, n_cpy = 0;
-    size_t n_ids = 0;
-    int tok_lo = -1, tok_hi = -1;
-    while (j < n_tasks && n_recs < kSlotRecs) {
-      const int t = task_ids[j];
-      const int c = indptr[j + 1] - indptr[j];
-      int remaining = c - done_in_task;
-      if (remaining == 0) { ++j; done_in_task = 0; continue; }
-      if (done_in_task == 0 && last_page_shared(kv, t)) {
-        // the task ends inside a page that others hold: give it a private copy before anything is written
-        if (n_ids == kSlotPageIds) break;
-        auto& pg0 = kv->pages[t];
-        const int32_t old_page = pg0.back(), new_page = pop_page(kv);
-        cpy_src[n_cpy] = old_page;
-        cpy_dst[n_cpy] = new_page;
-        ++n_cpy;
-        idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg0.size() - 1;
-        val[n_ids] = new_page;
-        ++n_ids;
-        pg0.back() = new_page;
-        unref_page(kv, old_page);
-      }
-      const int pos0 = kv->len[t];
-      // tokens that fit: up to the page-id budget of this upload
-      const int room_in_last = (int)((long long)ceil_div(pos0, g.S) * g.S - pos0);
-      const size_t ids_left = kSlotPageIds - n_ids;
-      long long can = room_in_last + (long long)ids_left * g.S;
-      if (can <= 0) break;
-      const int take = (int)std::min<long long>(remaining, can);
-      const int new_pages = ceil_div(pos0 + take, g.S) - ceil_div(pos0, g.S);
-      auto& pg = kv->pages[t];
-      for (int k = 0; k < new_pages; ++k) {
-        const int32_t page = pop_page(kv);
-        idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size();
-        val[n_ids] = page;
-        ++n_ids;
-        pg.push_back(page);
-      }
-      AppendRec& r = recs[n_recs++];
-      r.table_off = t * g.max_pages_per_task;
-      r.pos0 = pos0;
-      r.tok0 = indptr[j] + done_in_task;
-      r.count = take;
-      if (tok_lo < 0) tok_lo = r.tok0;
-      tok_hi = r.tok0 + take;
-      kv->len[t] += take;
-      kv->used_tokens += take;
-      done_in_task += take;
-      if (done_in_task == c) { ++j; done_in_task = 0; }
-      if (n_ids == kSlotPageIds) break;
-    }
-    if (n_recs == 0) continue;
-    // records hold absolute token indices; the kernel is launched over [tok_lo, tok_hi)
-    for (int k = 0; k < n_recs; ++k) recs[k].tok0 -= tok_lo;
-    // only the used prefixes of the three arrays (records, table indices, page ids) need to travel
-    if (cudaMemcpyAsync(slot->dev + 256, slot->host + 256, (size_t)n_recs * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return TIDE_ERR_CUDA;
+    idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
+    val = idx + kSlotPageIds;
+    cpy_src = val + kSlotPageIds;
+    cpy_dst = cpy_src + kSlotRecs;
+    return TIDE_OK;
+  };
+  auto flush = [&]() -> int {
+    if (slot == nullptr) return TIDE_OK;
     if (n_ids > 0) {
       uint8_t* didx = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec);
       if (cudaMemcpyAsync(didx, idx, n_ids * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
@@ -458,27 +448,152 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
         return TIDE_ERR_CUDA;
       ++kv->append_launches;
     }
-    if (n_cpy > 0) {
+    if (n_cpy > 0 && cow_out == nullptr) {
       uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
       if (cudaMemcpyAsync(dcpy, cpy_src, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
       if (cudaMemcpyAsync(dcpy + (size_t)kSlotRecs * 4, cpy_dst, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (launch_copy_pages(kv->pool, (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), n_cpy, g.page_bytes, st) != cudaSuccess)
+      for (int l = 0; l < kv->cfg.num_layers; ++l) {
+        if (launch_copy_pages(kv->layer_pool(l), (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), n_cpy,
+                              g.page_bytes, st) != cudaSuccess)
+          return TIDE_ERR_CUDA;
+        ++kv->append_launches;
+      }
+    }
+    const int r = release_slot(slot, st);
+    slot = nullptr;
+    n_ids = 0;
+    n_cpy = 0;
+    return r;
+  };
+  for (int j = 0; j < n_tasks; ++j) {
+    const int t = task_ids[j];
+    const int c = indptr[j + 1] - indptr[j];
+    if (c == 0) continue;
+    auto& pg = kv->pages[t];
+    if (last_page_shared(kv, t)) {
+      if ((rc = open_slot()) != TIDE_OK) return rc;
+      if (n_ids == kSlotPageIds || n_cpy == kSlotRecs) {
+        if ((rc = flush()) != TIDE_OK || (rc = open_slot()) != TIDE_OK) return rc;
+      }
+      const int32_t old_page = pg.back(), new_page = pop_page(kv);
+      if (cow_out != nullptr) {
+        cow_out->push_back(old_page);
+        cow_out->push_back(new_page);
+      }
+      cpy_src[n_cpy] = old_page;
+      cpy_dst[n_cpy] = new_page;
+      ++n_cpy;
+      idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size() - 1;
+      val[n_ids] = new_page;
+      ++n_ids;
+      pg.back() = new_page;
+      unref_page(kv, old_page);
+    }
+    const int new_pages = ceil_div(kv->len[t] + c, g.S) - ceil_div(kv->len[t], g.S);
+    for (int k = 0; k < new_pages; ++k) {
+      if ((rc = open_slot()) != TIDE_OK) return rc;
+      if (n_ids == kSlotPageIds) {
+        if ((rc = flush()) != TIDE_OK || (rc = open_slot()) != TIDE_OK) return rc;
+      }
+      const int32_t page = pop_page(kv);
+      idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size();
+      val[n_ids] = page;
+      ++n_ids;
+      pg.push_back(page);
+    }
+    kv->len[t] += c;
+    kv->used_tokens += c;
+  }
+  return flush();
+}
+
+// Writes the K/V rows of one layer into the LAST indptr[j+1]-indptr[j] positions of task_ids[j] (pure data; the
+// caller has checked that every task is at least that long).  Records travel in uploads of bounded size.
+static int write_tasks(tide_kv* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr,
+                       const void* new_k, const void* new_v, cudaStream_t st) {
+  const Geom& g = kv->g;
+  int j = 0;
+  int rc = TIDE_OK;
+  while (j < n_tasks) {
+    Slot* slot;
+    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+    AppendRec* recs = (AppendRec*)(slot->host + 256);
+    int n_recs = 0, tok_lo = -1, tok_hi = -1;
+    for (; j < n_tasks && n_recs < kSlotRecs; ++j) {
+      const int c = indptr[j + 1] - indptr[j];
+      if (c == 0) continue;
+      if (tok_lo < 0) tok_lo = indptr[j];
+      AppendRec& r = recs[n_recs++];
+      r.table_off = task_ids[j] * g.max_pages_per_task;
+      r.pos0 = kv->len[task_ids[j]] - c;
+      r.tok0 = indptr[j] - tok_lo;
+      r.count = c;
+      tok_hi = indptr[j + 1];
+    }
+    if (n_recs > 0) {
+      if (cudaMemcpyAsync(slot->dev + 256, recs, (size_t)n_recs * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return TIDE_ERR_CUDA;
+      AppendParams ap;
+      ap.pool = kv->layer_pool(layer);
+      ap.table = kv->d_table;
+      ap.recs = (const AppendRec*)(slot->dev + 256);
+      ap.n_recs = n_recs;
+      ap.n_tokens = tok_hi - tok_lo;
+      ap.new_k = (const uint16_t*)new_k + (size_t)tok_lo * g.Hkv * g.D;
+      ap.new_v = (const uint16_t*)new_v + (size_t)tok_lo * g.Hkv * g.D;
+      ap.g = g;
+      if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
       ++kv->append_launches;
     }
-    AppendParams ap;
-    ap.pool = kv->pool;
-    ap.table = kv->d_table;
-    ap.recs = (const AppendRec*)(slot->dev + 256);
-    ap.n_recs = n_recs;
-    ap.n_tokens = tok_hi - tok_lo;
-    ap.new_k = (const uint16_t*)new_k + (size_t)tok_lo * g.Hkv * g.D;
-    ap.new_v = (const uint16_t*)new_v + (size_t)tok_lo * g.Hkv * g.D;
-    ap.g = g;
-    if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
-    ++kv->append_launches;
     if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   }
+  return TIDE_OK;
+}
+
+static bool bad_kv_rows(int T, const void* new_k, const void* new_v) {
+  return T > 0 && (new_k == nullptr || new_v == nullptr || ((uintptr_t)new_k & 15) || ((uintptr_t)new_v & 15));
+}
+
+int tide_kv_extend(tide_kv_t* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, void* stream) {
+  if (kv == nullptr || n_tasks < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_tasks == 0) return TIDE_OK;
+  int rc = check_task_list(kv, n_tasks, task_ids, indptr);
+  if (rc != TIDE_OK) return rc;
+  kv->append_launches = 0;
+  return extend_tasks(kv, n_tasks, task_ids, indptr, (cudaStream_t)stream, nullptr);
+}
+
+int tide_kv_write(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr,
+                  const void* new_k, const void* new_v, void* stream) {
+  if (kv == nullptr || layer < 0 || layer >= kv->cfg.num_layers || n_tasks < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_tasks == 0) return TIDE_OK;
+  int rc = check_task_list(kv, n_tasks, task_ids, indptr);
+  if (rc != TIDE_OK) return rc;
+  if (bad_kv_rows(indptr[n_tasks], new_k, new_v)) return TIDE_ERR_INVALID_ARG;
+  for (int j = 0; j < n_tasks; ++j)
+    if (indptr[j + 1] - indptr[j] > kv->len[task_ids[j]]) return TIDE_ERR_CTX_RANGE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (kv->profiling) cudaEventRecord(kv->ev_append[0], st);
+  rc = write_tasks(kv, layer, n_tasks, task_ids, indptr, new_k, new_v, st);
+  if (rc == TIDE_OK && kv->profiling) {
+    cudaEventRecord(kv->ev_append[1], st);
+    kv->have_append_times = true;
+  }
+  return rc;
+}
+
+int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr,
+                   const void* new_k, const void* new_v, void* stream) {
+  if (kv == nullptr || layer != 0 || n_tasks < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_tasks == 0) return TIDE_OK;
+  int rc = check_task_list(kv, n_tasks, task_ids, indptr);
+  if (rc != TIDE_OK) return rc;
+  if (bad_kv_rows(indptr[n_tasks], new_k, new_v)) return TIDE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  kv->append_launches = 0;
+  if (kv->profiling) cudaEventRecord(kv->ev_append[0], st);
+  if ((rc = extend_tasks(kv, n_tasks, task_ids, indptr, st, nullptr)) != TIDE_OK) return rc;
+  if ((rc = write_tasks(kv, 0, n_tasks, task_ids, indptr, new_k, new_v, st)) != TIDE_OK) return rc;
   if (kv->profiling) {
     cudaEventRecord(kv->ev_append[1], st);
     kv->have_append_times = true;
@@ -487,12 +602,12 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
 }
 
 int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k, void* out_v, void* stream) {
-  if (kv == nullptr || layer != 0 || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
+  if (kv == nullptr || layer < 0 || layer >= kv->cfg.num_layers || !task_in_range(kv, task)) return TIDE_ERR_INVALID_ARG;
   if (!kv->live[task]) return TIDE_ERR_UNKNOWN_TASK;
   if (kv->len[task] == 0) return TIDE_OK;
   if (out_k == nullptr || out_v == nullptr || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15)) return TIDE_ERR_INVALID_ARG;
   const int32_t* row = kv->d_table + (size_t)task * kv->g.max_pages_per_task;
-  if (launch_read(kv->pool, row, 0, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
+  if (launch_read(kv->layer_pool(layer), row, 0, kv->len[task], (uint16_t*)out_k, (uint16_t*)out_v, kv->g, (cudaStream_t)stream) != cudaSuccess)
     return TIDE_ERR_CUDA;
   return TIDE_OK;
 }
@@ -545,8 +660,10 @@ int tide_kv_fork(tide_kv_t* kv, int32_t layer, int32_t parent, int32_t child, vo
       uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
       if (cudaMemcpyAsync(dcpy, hc, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
       if (cudaMemcpyAsync(dcpy + (size_t)kSlotRecs * 4, hc + kSlotRecs, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (launch_copy_pages(kv->pool, (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), 1, g.page_bytes, st) != cudaSuccess)
-        return TIDE_ERR_CUDA;
+      for (int l = 0; l < kv->cfg.num_layers; ++l)
+        if (launch_copy_pages(kv->layer_pool(l), (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), 1, g.page_bytes,
+                              st) != cudaSuccess)
+          return TIDE_ERR_CUDA;
     }
     if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   }
@@ -592,34 +709,72 @@ int tide_kv_prune(tide_kv_t* kv, int32_t layer, int32_t task, int32_t keep_prefi
   const int tail = len - tail_begin;
   if (tail_begin == keep_prefix) return TIDE_OK;   // nothing is dropped
   const Geom& g = kv->g;
+  const auto& pg = kv->pages[task];
+  // ---- validation: the pages the shorter task needs must be there once the dropped ones are back ----
+  const int kept = ceil_div(keep_prefix, g.S);              // pages that stay in the table
+  const int first = keep_prefix / g.S;                      // first page that is dropped or written again
+  bool shared_any = false;
+  long long freed = 0;
+  for (size_t i = (size_t)first; i < pg.size(); ++i) {
+    const bool shared = kv->refcnt[(size_t)pg[i]] > 1;
+    shared_any = shared_any || shared;
+    if ((int)i >= kept && !shared) ++freed;
+  }
+  long long need = ceil_div(keep_prefix + tail, g.S) - kept;
+  if (tail > 0 && keep_prefix % g.S != 0 && kv->refcnt[(size_t)pg[(size_t)first]] > 1) ++need;
+  if (need > (long long)kv->free_stack.size() + freed) return TIDE_ERR_NO_PAGES;
+  const int chunk_cap = (int)std::min<int64_t>(kv->cfg.max_batch_tokens, 0x7fffffff);
+  // A task that shares none of these pages gets the same pages back in the same places, so its tail can move in
+  // place, chunk by chunk.  Otherwise its new pages differ from the old ones and may be old ones in other places:
+  // the whole tail of a layer has to sit in the staging area before anything of that layer is written.
+  if (shared_any && tail > chunk_cap) return TIDE_ERR_WORKSPACE;
+
   cudaStream_t st = (cudaStream_t)stream;
   uint16_t* sk = (uint16_t*)(kv->ws + kv->lay.off_stage_k);
   uint16_t* sv = (uint16_t*)(kv->ws + kv->lay.off_stage_v);
-  const int chunk_cap = (int)std::min<int64_t>(kv->cfg.max_batch_tokens, 0x7fffffff);
-  // The shorter task needs no more pages than it holds, and truncate returns pages in the order in which the
-  // appends below take them again, so the kept part of the table does not change and nothing can fail below.
-  int rc = tide_kv_truncate(kv, task, keep_prefix);
-  if (rc != TIDE_OK) return rc;
   const int32_t* row = kv->d_table + (size_t)task * g.max_pages_per_task;
-  // Move the tail down in chunks, front to back: a chunk is written below the positions the next one reads.
-  for (int done = 0; done < tail; done += chunk_cap) {
-    const int n = std::min(chunk_cap, tail - done);
-    if (launch_read(kv->pool, row, tail_begin + done, n, sk, sv, g, st) != cudaSuccess) return TIDE_ERR_CUDA;
-    const int32_t ip[2] = {0, n};
-    rc = tide_kv_append(kv, layer, 1, &task, ip, sk, sv, stream);
-    if (rc != TIDE_OK) return rc;
+  const int L = kv->cfg.num_layers;
+  int rc;
+  if (!shared_any) {
+    if ((rc = tide_kv_truncate(kv, task, keep_prefix)) != TIDE_OK) return rc;
+    // front to back: a chunk is written below the positions the next one reads
+    for (int done = 0; done < tail; done += chunk_cap) {
+      const int n = std::min(chunk_cap, tail - done);
+      const int32_t ip[2] = {0, n};
+      if ((rc = extend_tasks(kv, 1, &task, ip, st, nullptr)) != TIDE_OK) return rc;
+      for (int l = 0; l < L; ++l) {
+        if (launch_read(kv->layer_pool(l), row, tail_begin + done, n, sk, sv, g, st) != cudaSuccess) return TIDE_ERR_CUDA;
+        if ((rc = write_tasks(kv, l, 1, &task, ip, sk, sv, st)) != TIDE_OK) return rc;
+      }
+    }
+    return TIDE_OK;
+  }
+  // keep the row as it is now: the tail is read through it after the table has changed
+  if (cudaMemcpyAsync(kv->d_old_row, row, pg.size() * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  if ((rc = tide_kv_truncate(kv, task, keep_prefix)) != TIDE_OK) return rc;
+  const int32_t ip[2] = {0, tail};
+  std::vector<int32_t> cow;
+  if ((rc = extend_tasks(kv, 1, &task, ip, st, &cow)) != TIDE_OK) return rc;
+  const int32_t *d_src = nullptr, *d_dst = nullptr;
+  if (!cow.empty()) {
+    // the one (old, new) pair sits behind the saved row; the source is pageable, so the call returns with it staged
+    int32_t* d_pair = kv->d_old_row + g.max_pages_per_task;
+    if (cudaMemcpyAsync(d_pair, cow.data(), 8, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    d_src = d_pair;
+    d_dst = d_pair + 1;
+  }
+  for (int l = 0; l < L; ++l) {
+    if (launch_read(kv->layer_pool(l), kv->d_old_row, tail_begin, tail, sk, sv, g, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (d_src != nullptr && launch_copy_pages(kv->layer_pool(l), d_src, d_dst, 1, g.page_bytes, st) != cudaSuccess)
+      return TIDE_ERR_CUDA;
+    if ((rc = write_tasks(kv, l, 1, &task, ip, sk, sv, st)) != TIDE_OK) return rc;
   }
   return TIDE_OK;
 }
 
-int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows, const int32_t* page_table,
-                const void* q, float scale, void* out, float* lse, void* stream) {
-  if (kv == nullptr || layer != 0 || n_rows < 0) return TIDE_ERR_INVALID_ARG;
-  if (n_rows == 0) return TIDE_OK;
-  if (rows == nullptr || q == nullptr || out == nullptr) return TIDE_ERR_INVALID_ARG;
-  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)lse & 3) || ((uintptr_t)page_table & 3)) return TIDE_ERR_INVALID_ARG;
-  if (!(scale == scale) || n_rows > kv->cfg.max_batch_rows) return n_rows > kv->cfg.max_batch_rows ? TIDE_ERR_WORKSPACE : TIDE_ERR_INVALID_ARG;
-  const Geom& g = kv->g;
+// Row checks of every attention call: live tasks, 1 <= q_len <= ctx_len <= resident length, batch limits.
+static int check_rows(tide_kv* kv, int32_t n_rows, const tide_row_t* rows) {
+  if (n_rows > kv->cfg.max_batch_rows) return TIDE_ERR_WORKSPACE;
   long long total_q = 0;
   for (int b = 0; b < n_rows; ++b) {
     const tide_row_t& r = rows[b];
@@ -629,44 +784,43 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
     total_q += r.q_len;
   }
   if (total_q > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
+  return TIDE_OK;
+}
 
-  // ---- plan: one segment per row, decode-style (<= 16 packed rows) or tile-style ----
+// The work plan of one batch: one segment per row, decode-style (<= 16 packed rows), warp-MMA tile-style or
+// tcgen05-style; long contexts are split along the keys so that the grid has about items_per_sm items per SM.
+// The plan depends on the rows only, so every layer of a step can use it.
+static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool umma_ok, PlanHost& P) {
+  const Geom& g = kv->g;
   enum { kDec = 0, kTile = 1, kUmma = 2 };
-  struct RowPlan { int b; int kind; int n_mtiles; long long items; };
-  const bool umma_ok = g.D == 128 && scale > 0.f;
+  struct RowPlan { int kind; int n_mtiles; long long items; };
   std::vector<RowPlan> plan((size_t)n_rows);
   long long w_dec = 0, w_tile = 0, items_tile_nosplit = 0;
-  {
-    for (int b = 0; b < n_rows; ++b) {
-      const tide_row_t& r = rows[b];
-      const int R = r.q_len * g.G;
-      RowPlan& p = plan[(size_t)b];
-      p.b = b;
-      p.kind = R <= kDecodeTileRows ? kDec : (umma_ok && R >= kv->umma_min_rows ? kUmma : kTile);
-      p.n_mtiles = p.kind == kDec ? 1 : ceil_div(R, p.kind == kUmma ? 2 * kUmmaTileRows : kMmaTileRows);
-      p.items = (long long)g.Hkv * p.n_mtiles;
-      if (p.kind == kDec) w_dec += (long long)g.Hkv * r.ctx_len;
-      else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
-    }
+  for (int b = 0; b < n_rows; ++b) {
+    const tide_row_t& r = rows[b];
+    const int R = r.q_len * g.G;
+    RowPlan& p = plan[(size_t)b];
+    p.kind = R <= kDecodeTileRows ? kDec : (umma_ok && R >= kv->umma_min_rows ? kUmma : kTile);
+    p.n_mtiles = p.kind == kDec ? 1 : ceil_div(R, p.kind == kUmma ? 2 * kUmmaTileRows : kMmaTileRows);
+    p.items = (long long)g.Hkv * p.n_mtiles;
+    if (p.kind == kDec) w_dec += (long long)g.Hkv * r.ctx_len;
+    else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
   }
   const long long target = (long long)kNumSms * kv->items_per_sm;
   long long chunk_dec = std::max<long long>(256, align_up((size_t)(w_dec / target + 1), kStageKeys));
   long long chunk_tile = (items_tile_nosplit >= target / 2)
                              ? (1LL << 30)
                              : std::max<long long>(2048, align_up((size_t)(w_tile / target + 1), kStageKeys));
-  std::vector<Segment> seg_dec, seg_tile, seg_umma, seg_merge;
-  long long items_dec = 0, items_tile = 0, items_umma = 0, part_rows = 0, merge_rows = 0;
   for (int attempt = 0; attempt < 40; ++attempt) {
-    seg_dec.clear(); seg_tile.clear(); seg_umma.clear();
-    part_rows = 0;
-    long long qoff = 0;
+    P.seg_dec.clear(); P.seg_tile.clear(); P.seg_umma.clear();
+    long long part_rows = 0, qoff = 0;
     for (int b = 0; b < n_rows; ++b) {
       const tide_row_t& r = rows[b];
       const RowPlan& p = plan[(size_t)b];
       const long long chunk_target = p.kind == kDec ? chunk_dec : chunk_tile;
       int n_splits = (int)std::min<long long>(kMaxSplits, ((long long)r.ctx_len + chunk_target - 1) / chunk_target);
       n_splits = std::max(1, n_splits);
-      int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), 2 * kStageKeys);
+      const int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), 2 * kStageKeys);
       n_splits = ceil_div(r.ctx_len, chunk);
       Segment s{};
       s.table_off = r.task * g.max_pages_per_task;
@@ -678,7 +832,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
       s.chunk = chunk;
       s.part_base = 0;
       if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
-      (p.kind == kDec ? seg_dec : p.kind == kTile ? seg_tile : seg_umma).push_back(s);
+      (p.kind == kDec ? P.seg_dec : p.kind == kTile ? P.seg_tile : P.seg_umma).push_back(s);
       qoff += r.q_len;
     }
     if (part_rows <= kv->lay.part_rows) break;
@@ -690,11 +844,13 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   auto heavier = [](const Segment& a, const Segment& b) {
     return std::min(a.chunk, a.p + a.n) > std::min(b.chunk, b.p + b.n);
   };
-  std::stable_sort(seg_dec.begin(), seg_dec.end(), heavier);
-  std::stable_sort(seg_tile.begin(), seg_tile.end(), heavier);
-  std::stable_sort(seg_umma.begin(), seg_umma.end(), heavier);
+  std::stable_sort(P.seg_dec.begin(), P.seg_dec.end(), heavier);
+  std::stable_sort(P.seg_tile.begin(), P.seg_tile.end(), heavier);
+  std::stable_sort(P.seg_umma.begin(), P.seg_umma.end(), heavier);
+  P.seg_merge.clear();
+  P.merge_rows = 0;
   long long part_cursor = 0;
-  for (auto* v : {&seg_dec, &seg_tile, &seg_umma}) {
+  for (auto* v : {&P.seg_dec, &P.seg_tile, &P.seg_umma}) {
     long long base = 0;
     for (Segment& s : *v) {
       s.item_base = (int32_t)base;
@@ -703,30 +859,36 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
       if (s.n_splits > 1) {
         s.part_base = (int32_t)part_cursor;
         part_cursor += (long long)s.n_splits * s.n * g.Hq;
-        s.merge_base = (int32_t)merge_rows;
-        merge_rows += (long long)s.n * g.Hq;
-        seg_merge.push_back(s);
+        s.merge_base = (int32_t)P.merge_rows;
+        P.merge_rows += (long long)s.n * g.Hq;
+        P.seg_merge.push_back(s);
       }
     }
-    (v == &seg_dec ? items_dec : v == &seg_tile ? items_tile : items_umma) = base;
+    (v == &P.seg_dec ? P.items_dec : v == &P.seg_tile ? P.items_tile : P.items_umma) = base;
   }
-  const size_t n_all = seg_dec.size() + seg_tile.size() + seg_umma.size() + seg_merge.size();
-  if (n_all * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
+  return TIDE_OK;
+}
 
-  cudaStream_t st = (cudaStream_t)stream;
-  Slot* slot;
-  int rc;
-  if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
-  Segment* h = (Segment*)(slot->host + 256);
-  std::copy(seg_dec.begin(), seg_dec.end(), h);
-  std::copy(seg_tile.begin(), seg_tile.end(), h + seg_dec.size());
-  std::copy(seg_umma.begin(), seg_umma.end(), h + seg_dec.size() + seg_tile.size());
-  std::copy(seg_merge.begin(), seg_merge.end(), h + seg_dec.size() + seg_tile.size() + seg_umma.size());
-  if (cudaMemcpyAsync(slot->dev + 256, h, n_all * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-  const Segment* d = (const Segment*)(slot->dev + 256);
+// Writes the four segment arrays one after the other at `h` and describes them as they will sit at `d`.
+static PlanDev pack_plan(const PlanHost& P, Segment* h, const Segment* d) {
+  Segment* w = h;
+  w = std::copy(P.seg_dec.begin(), P.seg_dec.end(), w);
+  w = std::copy(P.seg_tile.begin(), P.seg_tile.end(), w);
+  w = std::copy(P.seg_umma.begin(), P.seg_umma.end(), w);
+  std::copy(P.seg_merge.begin(), P.seg_merge.end(), w);
+  PlanDev pd;
+  pd.segs = d;
+  pd.n_dec = P.seg_dec.size(); pd.n_tile = P.seg_tile.size(); pd.n_umma = P.seg_umma.size(); pd.n_merge = P.seg_merge.size();
+  pd.items_dec = P.items_dec; pd.items_tile = P.items_tile; pd.items_umma = P.items_umma; pd.merge_rows = P.merge_rows;
+  return pd;
+}
 
+// The attention launches of one planned batch on one layer: kernel launches only (and, with `events`, the phase
+// time stamps), so a caller may capture them in a CUDA graph.
+static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32_t* page_table, const void* q, float scale,
+                       void* out, float* lse, cudaStream_t st, bool events, int64_t* n_launches) {
   AttendParams ap;
-  ap.pool = kv->pool;
+  ap.pool = kv->layer_pool(layer);
   ap.table = page_table ? page_table : kv->d_table;
   ap.q = (const uint16_t*)q;
   ap.out = (uint16_t*)out;
@@ -735,46 +897,148 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   ap.part_lse = kv->d_part_lse;
   ap.scale_log2e = scale * 1.4426950408889634f;
   ap.status = kv->d_status;
-  ap.g = g;
+  ap.g = kv->g;
   int64_t launches = 0;
-  if (kv->profiling) cudaEventRecord(kv->ev_attend[0], st);
-  if (items_dec > 0) {
-    ap.segs = d; ap.n_segs = (int)seg_dec.size(); ap.n_items = (int)items_dec;
+  if (events) cudaEventRecord(kv->ev_attend[0], st);
+  if (d.items_dec > 0) {
+    ap.segs = d.segs; ap.n_segs = (int)d.n_dec; ap.n_items = (int)d.items_dec;
     if (launch_attend_decode(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
-  if (kv->profiling) cudaEventRecord(kv->ev_attend[1], st);
-  if (items_tile > 0) {
-    ap.segs = d + seg_dec.size(); ap.n_segs = (int)seg_tile.size(); ap.n_items = (int)items_tile;
+  if (events) cudaEventRecord(kv->ev_attend[1], st);
+  if (d.items_tile > 0) {
+    ap.segs = d.segs + d.n_dec; ap.n_segs = (int)d.n_tile; ap.n_items = (int)d.items_tile;
     if (launch_attend_tile(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
-  if (items_umma > 0) {
-    ap.segs = d + seg_dec.size() + seg_tile.size(); ap.n_segs = (int)seg_umma.size(); ap.n_items = (int)items_umma;
+  if (d.items_umma > 0) {
+    ap.segs = d.segs + d.n_dec + d.n_tile; ap.n_segs = (int)d.n_umma; ap.n_items = (int)d.items_umma;
     if (launch_attend_umma(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
-  if (kv->profiling) cudaEventRecord(kv->ev_attend[2], st);
-  if (merge_rows > 0) {
+  if (events) cudaEventRecord(kv->ev_attend[2], st);
+  if (d.merge_rows > 0) {
     MergeParams mp;
-    mp.segs = d + seg_dec.size() + seg_tile.size() + seg_umma.size();
-    mp.n_segs = (int)seg_merge.size();
-    mp.n_rows = (int)merge_rows;
+    mp.segs = d.segs + d.n_dec + d.n_tile + d.n_umma;
+    mp.n_segs = (int)d.n_merge;
+    mp.n_rows = (int)d.merge_rows;
     mp.part_o = kv->d_part_o; mp.part_lse = kv->d_part_lse;
-    mp.out = (uint16_t*)out; mp.lse = lse; mp.Hq = g.Hq; mp.D = g.D;
+    mp.out = (uint16_t*)out; mp.lse = lse; mp.Hq = kv->g.Hq; mp.D = kv->g.D;
     if (launch_merge(mp, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
-  if (kv->profiling) {
+  if (events) {
     cudaEventRecord(kv->ev_attend[3], st);
     kv->have_attend_times = true;
   }
+  *n_launches = launches;
+  return TIDE_OK;
+}
+
+int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows, const int32_t* page_table,
+                const void* q, float scale, void* out, float* lse, void* stream) {
+  if (kv == nullptr || layer < 0 || layer >= kv->cfg.num_layers || n_rows < 0) return TIDE_ERR_INVALID_ARG;
+  if (n_rows == 0) return TIDE_OK;
+  if (rows == nullptr || q == nullptr || out == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)lse & 3) || ((uintptr_t)page_table & 3)) return TIDE_ERR_INVALID_ARG;
+  if (!(scale == scale)) return TIDE_ERR_INVALID_ARG;
+  int rc = check_rows(kv, n_rows, rows);
+  if (rc != TIDE_OK) return rc;
+  PlanHost P;
+  if ((rc = build_plan(kv, n_rows, rows, kv->g.D == 128 && scale > 0.f, P)) != TIDE_OK) return rc;
+  if (P.n_all() * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  Slot* slot;
+  if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+  const PlanDev pd = pack_plan(P, (Segment*)(slot->host + 256), (const Segment*)(slot->dev + 256));
+  if (cudaMemcpyAsync(slot->dev + 256, slot->host + 256, P.n_all() * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TIDE_ERR_CUDA;
+  int64_t launches = 0;
+  if ((rc = launch_plan(kv, layer, pd, page_table, q, scale, out, lse, st, kv->profiling, &launches)) != TIDE_OK) return rc;
   if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
-  kv->last_decode_items = items_dec;
-  kv->last_prefill_items = items_tile + items_umma;
-  kv->last_merge_rows = merge_rows;
+  kv->last_decode_items = pd.items_dec;
+  kv->last_prefill_items = pd.items_tile + pd.items_umma;
+  kv->last_merge_rows = pd.merge_rows;
   kv->last_launches = launches + kv->append_launches;
   kv->append_launches = 0;
+  return TIDE_OK;
+}
+
+int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void* stream) {
+  if (kv == nullptr || n_rows < 0) return TIDE_ERR_INVALID_ARG;
+  kv->step_valid = false;
+  if (n_rows == 0) return TIDE_OK;
+  if (rows == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (n_rows > kv->cfg.max_batch_rows) return TIDE_ERR_WORKSPACE;
+  const Geom& g = kv->g;
+  std::vector<int32_t> ids((size_t)n_rows), indptr((size_t)n_rows + 1);
+  indptr[0] = 0;
+  for (int b = 0; b < n_rows; ++b) {
+    const tide_row_t& r = rows[b];
+    if (!task_in_range(kv, r.task)) return TIDE_ERR_INVALID_ARG;
+    if (!kv->live[r.task]) return TIDE_ERR_UNKNOWN_TASK;
+    if (r.q_len < 1 || (long long)kv->len[r.task] + r.q_len != r.ctx_len) return TIDE_ERR_CTX_RANGE;
+    ids[(size_t)b] = r.task;
+    if ((long long)indptr[(size_t)b] + r.q_len > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
+    indptr[(size_t)b + 1] = indptr[(size_t)b] + r.q_len;
+  }
+  int rc = check_task_list(kv, n_rows, ids.data(), indptr.data());
+  if (rc != TIDE_OK) return rc;
+  // The plan needs the lengths after the step only through ctx_len, which the rows already carry, so it is built
+  // (and can still be refused) before anything changes.
+  PlanHost P;
+  if ((rc = build_plan(kv, n_rows, rows, g.D == 128, P)) != TIDE_OK) return rc;
+  if (kv->lay.step_seg_off + P.n_all() * sizeof(Segment) > kv->lay.step_bytes) return TIDE_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  kv->append_launches = 0;
+  if ((rc = extend_tasks(kv, n_rows, ids.data(), indptr.data(), st, nullptr)) != TIDE_OK) return rc;
+  // one upload: the write records of the rows, then the segments
+  if (kv->step_upload_pending && cudaEventSynchronize(kv->ev_step) != cudaSuccess) return TIDE_ERR_CUDA;
+  AppendRec* recs = (AppendRec*)kv->h_step;
+  for (int b = 0; b < n_rows; ++b) {
+    recs[b].table_off = rows[b].task * g.max_pages_per_task;
+    recs[b].pos0 = rows[b].ctx_len - rows[b].q_len;
+    recs[b].tok0 = indptr[(size_t)b];
+    recs[b].count = rows[b].q_len;
+  }
+  uint8_t* d_step = kv->ws + kv->lay.off_step;
+  kv->step_plan = pack_plan(P, (Segment*)(kv->h_step + kv->lay.step_seg_off), (const Segment*)(d_step + kv->lay.step_seg_off));
+  if (cudaMemcpyAsync(d_step, kv->h_step, kv->lay.step_seg_off + P.n_all() * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TIDE_ERR_CUDA;
+  if (cudaEventRecord(kv->ev_step, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  kv->step_upload_pending = true;
+  kv->step_recs = n_rows;
+  kv->step_tokens = indptr[(size_t)n_rows];
+  kv->step_valid = true;
+  kv->last_decode_items = P.items_dec;
+  kv->last_prefill_items = P.items_tile + P.items_umma;
+  kv->last_merge_rows = P.merge_rows;
+  return TIDE_OK;
+}
+
+int tide_step_layer(tide_kv_t* kv, int32_t layer, const void* new_k, const void* new_v, const void* q, float scale,
+                    void* out, float* lse, void* stream) {
+  if (kv == nullptr || layer < 0 || layer >= kv->cfg.num_layers) return TIDE_ERR_INVALID_ARG;
+  if (!kv->step_valid) return TIDE_ERR_INVALID_ARG;
+  if (q == nullptr || out == nullptr || bad_kv_rows(kv->step_tokens, new_k, new_v)) return TIDE_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)lse & 3)) return TIDE_ERR_INVALID_ARG;
+  if (!(scale > 0.f) || !(scale <= 3.0e38f)) return TIDE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  AppendParams ap;
+  ap.pool = kv->layer_pool(layer);
+  ap.table = kv->d_table;
+  ap.recs = (const AppendRec*)(kv->ws + kv->lay.off_step);
+  ap.n_recs = kv->step_recs;
+  ap.n_tokens = kv->step_tokens;
+  ap.new_k = (const uint16_t*)new_k;
+  ap.new_v = (const uint16_t*)new_v;
+  ap.g = kv->g;
+  if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  int64_t launches = 0;
+  const int rc = launch_plan(kv, layer, kv->step_plan, nullptr, q, scale, out, lse, st, false, &launches);
+  if (rc != TIDE_OK) return rc;
+  kv->last_launches = launches + 1;
   return TIDE_OK;
 }
 

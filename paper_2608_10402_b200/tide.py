@@ -47,6 +47,7 @@ EXPORTS = [
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
     "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune", "tide_kv_fork", "tide_kv_page_refs",
+    "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -100,9 +101,9 @@ def rows_array(rows):
     return arr
 
 
-def make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens):
+def make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens, num_layers=1):
     cfg = tide_kv_config_t()
-    cfg.num_layers = 1
+    cfg.num_layers = int(num_layers)
     cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.page_size = int(Hq), int(Hkv), int(D), int(S)
     cfg.max_tasks, cfg.max_pages_per_task, cfg.max_batch_rows = int(max_tasks), int(max_pages_per_task), int(max_batch_rows)
     cfg.num_pages, cfg.max_batch_tokens = int(num_pages), int(max_batch_tokens)
@@ -119,9 +120,11 @@ class TideKV:
     """One paged cache on the current CUDA device.  Methods mirror the C entry points one to one."""
 
     def __init__(self, Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens,
-                 free_order=None, device="cuda"):
+                 free_order=None, device="cuda", num_layers=1):
         import torch
-        self.cfg = make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens)
+        self.cfg = make_config(Hq, Hkv, D, S, num_pages, max_tasks, max_pages_per_task, max_batch_rows, max_batch_tokens,
+                               num_layers)
+        self.num_layers = int(num_layers)
         pb, wb = tide_kv_required_bytes(self.cfg)
         # PyTorch only supplies device memory (and streams)
         self.pool = torch.empty(pb + 1024, dtype=torch.uint8, device=device)
@@ -185,9 +188,28 @@ class TideKV:
         _check(lib.tide_kv_append(self.handle, ctypes.c_int32(0), ctypes.c_int32(ids.shape[0]), _ptr(ids), _ptr(ip),
                                   _ptr(new_k), _ptr(new_v), _stream(stream)), "tide_kv_append")
 
-    def attend(self, rows, q, scale, out, lse=None, page_table=None, stream=None):
+    def extend(self, task_ids, indptr, stream=None):
+        ids, ip = _i32(task_ids), _i32(indptr)
+        assert ip.shape[0] == ids.shape[0] + 1
+        _check(lib.tide_kv_extend(self.handle, ctypes.c_int32(ids.shape[0]), _ptr(ids), _ptr(ip), _stream(stream)), "tide_kv_extend")
+
+    def write(self, layer, task_ids, indptr, new_k, new_v, stream=None):
+        ids, ip = _i32(task_ids), _i32(indptr)
+        assert ip.shape[0] == ids.shape[0] + 1
+        _check(lib.tide_kv_write(self.handle, ctypes.c_int32(layer), ctypes.c_int32(ids.shape[0]), _ptr(ids), _ptr(ip),
+                                 _ptr(new_k), _ptr(new_v), _stream(stream)), "tide_kv_write")
+
+    def step_begin(self, rows, stream=None):
         arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
-        _check(lib.tide_attend(self.handle, ctypes.c_int32(0), ctypes.c_int32(len(arr)), arr, _ptr(page_table), _ptr(q),
+        _check(lib.tide_step_begin(self.handle, ctypes.c_int32(len(arr)), arr, _stream(stream)), "tide_step_begin")
+
+    def step_layer(self, layer, new_k, new_v, q, scale, out, lse=None, stream=None):
+        _check(lib.tide_step_layer(self.handle, ctypes.c_int32(layer), _ptr(new_k), _ptr(new_v), _ptr(q),
+                                   ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)), "tide_step_layer")
+
+    def attend(self, rows, q, scale, out, lse=None, page_table=None, stream=None, layer=0):
+        arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
+        _check(lib.tide_attend(self.handle, ctypes.c_int32(layer), ctypes.c_int32(len(arr)), arr, _ptr(page_table), _ptr(q),
                                ctypes.c_float(scale), _ptr(out), _ptr(lse), _stream(stream)), "tide_attend")
 
     def attend_decode_static(self, rows, q, scale, out, lse=None, stream=None):
@@ -219,13 +241,13 @@ class TideKV:
         _check(lib.tide_kv_usage(self.handle, ctypes.byref(u), ctypes.byref(f)), "tide_kv_usage")
         return u.value, f.value
 
-    def read(self, task, stream=None):
+    def read(self, task, stream=None, layer=0):
         """Logical K, V of a task as torch uint16-bit tensors (int16 view) [len, Hkv, D] on the device."""
         import torch
         L = self.task_len(task)
         k = torch.empty((L, self.Hkv, self.D), dtype=torch.int16, device=self.pool.device)
         v = torch.empty_like(k)
-        _check(lib.tide_kv_read(self.handle, ctypes.c_int32(0), ctypes.c_int32(task), _ptr(k), _ptr(v), _stream(stream)), "tide_kv_read")
+        _check(lib.tide_kv_read(self.handle, ctypes.c_int32(layer), ctypes.c_int32(task), _ptr(k), _ptr(v), _stream(stream)), "tide_kv_read")
         return k, v
 
     def status(self, stream=None):
