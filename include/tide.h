@@ -139,7 +139,10 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
  * tokens to every row's task (rows must name distinct tasks; ctx_len must equal the resident length
  * after the append), attends, and copies out / lse back.  new_k, new_v: host bf16 [sum q_len, Hkv, D];
  * q, out: host bf16 [sum q_len, Hq, D]; lse: host fp32 or NULL.  Host buffers should be pinned for
- * the copies to be asynchronous.  The call returns after the results have arrived. */
+ * the copies to be asynchronous.  The call returns after the results have arrived.  A large step is cut
+ * into groups of consecutive rows whose copies (on two streams the library owns) run beside the kernels
+ * of other groups; pages, cache contents and results do not depend on the cut.  The whole step is checked
+ * (rows, duplicates, pages) before anything is copied or changed.  Takes layer 0 only. */
 int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* rows /*host*/,
                    const void* new_k /*host*/, const void* new_v /*host*/, const void* q /*host*/,
                    float scale, void* out /*host*/, float* lse /*host or NULL*/, void* stream);

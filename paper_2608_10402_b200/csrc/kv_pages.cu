@@ -4,6 +4,8 @@
 // observation tokens' K/V rows are copied into the task's pages next to its preserved state, which
 // replaces re-running prefill over the history (Section 1, first challenge).  It is a pure bit copy,
 // bound by HBM bandwidth: 2 * Hkv * D * 2 bytes read and as many written per new token.
+#include <algorithm>
+
 #include "tide_internal.h"
 
 namespace tide {
@@ -17,6 +19,21 @@ __global__ void table_update_kernel(int32_t* __restrict__ table, const int32_t* 
 cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   table_update_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, idx, val, n);
+  return cudaGetLastError();
+}
+
+// Small host-to-device upload done by the SMs: src is pinned host memory mapped into the device's address space.
+// Unlike a copy-engine transfer it does not queue behind large copies that other streams have in flight.
+__global__ void upload_kernel(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, size_t n_words) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+cudaError_t launch_upload(void* dst, const void* src_mapped_host, size_t bytes, cudaStream_t s) {
+  if (bytes == 0) return cudaSuccess;
+  const size_t n = bytes / 4;
+  const unsigned blocks = (unsigned)std::min<size_t>((n + 255) / 256, 64);
+  upload_kernel<<<blocks, 256, 0, s>>>((uint32_t*)dst, (const uint32_t*)src_mapped_host, n);
   return cudaGetLastError();
 }
 

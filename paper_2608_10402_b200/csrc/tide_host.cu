@@ -18,12 +18,14 @@ using namespace tide;
 
 namespace {
 
-constexpr int kSlots = 4;                    // staging ring depth
+constexpr int kSlots = 8;                    // staging ring depth
 constexpr size_t kSlotPageIds = 64 * 1024;   // most new page ids per upload
 constexpr int kSlotRecs = 2048;              // most append records per upload
 constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
 constexpr int kNumSms = 148;
 constexpr long long kPartRowsBase = 256 * 1024;
+constexpr int kMaxHostChunks = 8;                 // most row groups of one host-buffer step
+constexpr size_t kHostChunkBytes = 64u << 20;      // transfer bytes per group from which cutting a step pays
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -101,6 +103,12 @@ struct tide_kv {
   bool step_upload_pending = false, step_valid = false;
   PlanDev step_plan;
   int step_recs = 0, step_tokens = 0;
+  // host-buffer steps: copy streams and the events that order them against the caller's stream
+  cudaStream_t st_in = nullptr, st_out = nullptr;
+  cudaEvent_t ev_host[2 * kMaxHostChunks + 2] = {};   // copies-in done, kernels done (per group); start, end
+  int host_step_chunks = 0;   // 0 = by size
+  bool slots_mapped = false;     // the staging slots' host addresses are valid on the device too
+  bool upload_by_kernel = false;
   uint8_t* layer_pool(int layer) const { return pool + (size_t)layer * layer_stride; }
 };
 
@@ -202,6 +210,13 @@ int acquire_slot(tide_kv* kv, Slot** out) {
   return TIDE_OK;
 }
 
+// Small upload of planning data from a staging slot.  Normally a copy-engine transfer; while a host-buffer step
+// has large copies in flight on other streams it is done by a kernel instead, which does not queue behind them.
+cudaError_t upload(const tide_kv* kv, void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  if (kv->upload_by_kernel) return launch_upload(dst, src, bytes, st);
+  return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
+}
+
 int release_slot(Slot* s, cudaStream_t st) {
   s->used = true;
   return cudaEventRecord(s->ev, st) == cudaSuccess ? TIDE_OK : TIDE_ERR_CUDA;
@@ -268,7 +283,13 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   ok = ok && cudaHostAlloc((void**)&kv->h_step, lay.step_bytes, cudaHostAllocDefault) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&kv->ev_step, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; ok && i < kSlots; ++i) {
-    ok = cudaHostAlloc((void**)&kv->slots[i].host, lay.slot_bytes, cudaHostAllocDefault) == cudaSuccess;
+    ok = cudaHostAlloc((void**)&kv->slots[i].host, lay.slot_bytes, cudaHostAllocMapped) == cudaSuccess;
+    void* on_device = nullptr;
+    if (ok && i == 0) kv->slots_mapped = true;
+    if (ok && (cudaHostGetDevicePointer(&on_device, kv->slots[i].host, 0) != cudaSuccess || on_device != (void*)kv->slots[i].host)) {
+      kv->slots_mapped = false;   // no unified addressing: uploads stay copy-engine transfers
+      cudaGetLastError();
+    }
     ok = ok && cudaEventCreateWithFlags(&kv->slots[i].ev, cudaEventDisableTiming) == cudaSuccess;
     kv->slots[i].dev = kv->ws + lay.off_meta + (size_t)i * lay.slot_bytes;
   }
@@ -282,6 +303,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->mark.assign((size_t)cfg->max_tasks, 0);
   kv->refcnt.assign((size_t)cfg->num_pages, 0);
   if (const char* e = getenv("TIDE_ITEMS_PER_SM")) kv->items_per_sm = std::max(1, atoi(e));  // tuning knob
+  if (const char* e = getenv("TIDE_HOST_STEP_CHUNKS")) kv->host_step_chunks = std::max(0, atoi(e));  // tuning knob
   if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
   *out = kv;
@@ -298,6 +320,9 @@ int tide_kv_destroy(tide_kv_t* kv) {
   if (kv->h_status) cudaFreeHost(kv->h_status);
   if (kv->h_step) cudaFreeHost(kv->h_step);
   if (kv->ev_step) cudaEventDestroy(kv->ev_step);
+  if (kv->st_in) cudaStreamDestroy(kv->st_in);
+  if (kv->st_out) cudaStreamDestroy(kv->st_out);
+  for (cudaEvent_t e : kv->ev_host) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : kv->ev_append) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : kv->ev_attend) if (e) cudaEventDestroy(e);
   delete kv;
@@ -403,13 +428,8 @@ static int check_task_list(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids
   return TIDE_OK;
 }
 
-// Grows task_ids[j] by indptr[j+1]-indptr[j] tokens: host tables first, then the device page table, in uploads of
-// bounded size.  No K/V is written.  A task that ends inside a page that other tasks hold gets a private copy of
-// that page before its other pages are taken: with cow_out == nullptr the copy runs here on every layer, otherwise
-// the (old, new) page pairs are handed back and the caller copies (it may have to read the old pages first).
-// The task list must have passed check_task_list.
-static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, cudaStream_t st,
-                        std::vector<int32_t>* cow_out) {
+// Would growing task_ids[j] by indptr[j+1]-indptr[j] tokens fit the page tables and the free stack?
+static int check_extend(const tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr) {
   const Geom& g = kv->g;
   long long need = 0;
   for (int j = 0; j < n_tasks; ++j) {
@@ -420,7 +440,19 @@ static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, c
     need += after - ceil_div(kv->len[t], g.S);
     if (c > 0 && last_page_shared(kv, t)) ++need;   // a private copy of the shared partial page comes first
   }
-  if (need > (long long)kv->free_stack.size()) return TIDE_ERR_NO_PAGES;
+  return need > (long long)kv->free_stack.size() ? TIDE_ERR_NO_PAGES : TIDE_OK;
+}
+
+// Grows task_ids[j] by indptr[j+1]-indptr[j] tokens: host tables first, then the device page table, in uploads of
+// bounded size.  No K/V is written.  A task that ends inside a page that other tasks hold gets a private copy of
+// that page before its other pages are taken: with cow_out == nullptr the copy runs here on every layer, otherwise
+// the (old, new) page pairs are handed back and the caller copies (it may have to read the old pages first).
+// The task list must have passed check_task_list.
+static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, cudaStream_t st,
+                        std::vector<int32_t>* cow_out) {
+  const Geom& g = kv->g;
+  int rc = check_extend(kv, n_tasks, task_ids, indptr);
+  if (rc != TIDE_OK) return rc;
 
   // ---- mutation ----
   kv->step_valid = false;
@@ -428,7 +460,6 @@ static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, c
   int32_t *idx = nullptr, *val = nullptr, *cpy_src = nullptr, *cpy_dst = nullptr;
   size_t n_ids = 0;
   int n_cpy = 0;
-  int rc = TIDE_OK;
   auto open_slot = [&]() -> int {
     if (slot != nullptr) return TIDE_OK;
     if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
@@ -442,16 +473,16 @@ static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, c
     if (slot == nullptr) return TIDE_OK;
     if (n_ids > 0) {
       uint8_t* didx = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec);
-      if (cudaMemcpyAsync(didx, idx, n_ids * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (cudaMemcpyAsync(didx + kSlotPageIds * 4, val, n_ids * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (upload(kv, didx, idx, n_ids * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (upload(kv, didx + kSlotPageIds * 4, val, n_ids * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
       if (launch_table_update(kv->d_table, (const int32_t*)didx, (const int32_t*)(didx + kSlotPageIds * 4), (int)n_ids, st) != cudaSuccess)
         return TIDE_ERR_CUDA;
       ++kv->append_launches;
     }
     if (n_cpy > 0 && cow_out == nullptr) {
       uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
-      if (cudaMemcpyAsync(dcpy, cpy_src, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (cudaMemcpyAsync(dcpy + (size_t)kSlotRecs * 4, cpy_dst, (size_t)n_cpy * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (upload(kv, dcpy, cpy_src, (size_t)n_cpy * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      if (upload(kv, dcpy + (size_t)kSlotRecs * 4, cpy_dst, (size_t)n_cpy * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
       for (int l = 0; l < kv->cfg.num_layers; ++l) {
         if (launch_copy_pages(kv->layer_pool(l), (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), n_cpy,
                               g.page_bytes, st) != cudaSuccess)
@@ -531,7 +562,7 @@ static int write_tasks(tide_kv* kv, int32_t layer, int32_t n_tasks, const int32_
       tok_hi = indptr[j + 1];
     }
     if (n_recs > 0) {
-      if (cudaMemcpyAsync(slot->dev + 256, recs, (size_t)n_recs * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      if (upload(kv, slot->dev + 256, recs, (size_t)n_recs * sizeof(AppendRec), st) != cudaSuccess)
         return TIDE_ERR_CUDA;
       AppendParams ap;
       ap.pool = kv->layer_pool(layer);
@@ -952,7 +983,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   Slot* slot;
   if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
   const PlanDev pd = pack_plan(P, (Segment*)(slot->host + 256), (const Segment*)(slot->dev + 256));
-  if (cudaMemcpyAsync(slot->dev + 256, slot->host + 256, P.n_all() * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (upload(kv, slot->dev + 256, slot->host + 256, P.n_all() * sizeof(Segment), st) != cudaSuccess)
     return TIDE_ERR_CUDA;
   int64_t launches = 0;
   if ((rc = launch_plan(kv, layer, pd, page_table, q, scale, out, lse, st, kv->profiling, &launches)) != TIDE_OK) return rc;
@@ -1060,6 +1091,10 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
     if ((long long)indptr[(size_t)b] + r.q_len > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
     indptr[(size_t)b + 1] = indptr[(size_t)b] + r.q_len;
   }
+  int rc = check_task_list(kv, n_rows, ids.data(), indptr.data());
+  if (rc == TIDE_OK) rc = check_extend(kv, n_rows, ids.data(), indptr.data());
+  if (rc != TIDE_OK) return rc;   // nothing has been copied or changed
+  if (!(scale == scale)) return TIDE_ERR_INVALID_ARG;
   const size_t T = (size_t)indptr[(size_t)n_rows];
   cudaStream_t st = (cudaStream_t)stream;
   uint8_t* dk = kv->ws + kv->lay.off_stage_k;
@@ -1067,18 +1102,83 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
   uint8_t* dq = kv->ws + kv->lay.off_stage_q;
   uint8_t* dout = kv->ws + kv->lay.off_stage_out;
   float* dlse = (float*)(kv->ws + kv->lay.off_stage_lse);
-  const size_t kv_bytes = T * g.Hkv * g.D * 2, q_bytes = T * g.Hq * g.D * 2;
-  // The copies only fill the staging area; tide_kv_append then validates everything (duplicates, pages)
-  // before it changes any state, so a rejected step leaves the cache as it was.
-  if (cudaMemcpyAsync(dk, new_k, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-  if (cudaMemcpyAsync(dv, new_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-  if (cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
-  int rc = tide_kv_append(kv, layer, n_rows, ids.data(), indptr.data(), dk, dv, stream);
-  if (rc != TIDE_OK) return rc;
-  rc = tide_attend(kv, layer, n_rows, rows, nullptr, dq, scale, dout, lse ? dlse : nullptr, stream);
-  if (rc != TIDE_OK) return rc;
-  if (cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TIDE_ERR_CUDA;
-  if (lse && cudaMemcpyAsync(lse, dlse, T * g.Hq * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  const size_t kv_row = (size_t)g.Hkv * g.D * 2, q_row = (size_t)g.Hq * g.D * 2, lse_row = (size_t)g.Hq * 4;
+  // Large steps are cut into groups of consecutive rows, each with its own copies in, append, attention and copies
+  // out, so that the transfers of one group run beside the kernels of another (copy engines in both directions
+  // and the SMs all busy).  Appending the groups in row order takes the same pages as one append of all rows.
+  const size_t bytes = T * (2 * kv_row + 2 * q_row + (lse ? lse_row : 0));
+  int n_chunks = kv->host_step_chunks > 0 ? kv->host_step_chunks : (int)std::min<size_t>(kMaxHostChunks, bytes / kHostChunkBytes);
+  n_chunks = std::max(1, std::min(std::min(n_chunks, kMaxHostChunks), n_rows));
+  if (n_chunks > 1 && kv->st_in == nullptr) {
+    bool ok = cudaStreamCreateWithFlags(&kv->st_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&kv->st_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 2 * kMaxHostChunks + 2; ++i)
+      ok = cudaEventCreateWithFlags(&kv->ev_host[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return TIDE_ERR_CUDA;
+  }
+  cudaStream_t s_in = n_chunks > 1 ? kv->st_in : st, s_out = n_chunks > 1 ? kv->st_out : st;
+  struct UploadMode {   // planning uploads bypass the copy engine while this step's large copies are in flight
+    tide_kv* kv;
+    ~UploadMode() { kv->upload_by_kernel = false; }
+  } upload_mode{kv};
+  kv->upload_by_kernel = n_chunks > 1 && kv->slots_mapped;
+  cudaEvent_t ev_start = kv->ev_host[2 * kMaxHostChunks], ev_end = kv->ev_host[2 * kMaxHostChunks + 1];
+  if (n_chunks > 1) {
+    // the copies in may not overtake work already queued on the caller's stream that still uses the staging area
+    if (cudaEventRecord(ev_start, st) != cudaSuccess || cudaStreamWaitEvent(s_in, ev_start, 0) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (cudaStreamWaitEvent(s_out, ev_start, 0) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  // rows [cut[c], cut[c+1]): up to the c+1-th share of the tokens, at least one row each
+  int cut[kMaxHostChunks + 1];
+  cut[0] = 0;
+  for (int c = 0; c < n_chunks; ++c) {
+    int r1 = cut[c] + 1;
+    const long long goal = (long long)T * (c + 1) / n_chunks;
+    while (r1 < n_rows && indptr[(size_t)r1 + 1] <= goal && n_rows - r1 > n_chunks - 1 - c) ++r1;
+    cut[c + 1] = c == n_chunks - 1 ? n_rows : r1;
+  }
+  // The copy engine works through its queue in order.  If the small uploads that every append and attention call
+  // makes (records, plan) go through the same queue, the copies in of group c+1 are queued right AFTER the calls
+  // of group c: queued earlier they would hold those uploads, and with them the kernels, back.
+  auto copy_in = [&](int c) -> int {
+    const size_t t0 = (size_t)indptr[(size_t)cut[c]], tn = (size_t)indptr[(size_t)cut[c + 1]] - t0;
+    if (cudaMemcpyAsync(dk + t0 * kv_row, (const uint8_t*)new_k + t0 * kv_row, tn * kv_row, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dv + t0 * kv_row, (const uint8_t*)new_v + t0 * kv_row, tn * kv_row, cudaMemcpyHostToDevice, s_in) != cudaSuccess ||
+        cudaMemcpyAsync(dq + t0 * q_row, (const uint8_t*)q + t0 * q_row, tn * q_row, cudaMemcpyHostToDevice, s_in) != cudaSuccess)
+      return TIDE_ERR_CUDA;
+    if (n_chunks > 1 && cudaEventRecord(kv->ev_host[c], s_in) != cudaSuccess) return TIDE_ERR_CUDA;
+    return TIDE_OK;
+  };
+  // With kernel uploads nothing of the calls goes through the copy engine, and every copy in can be queued at once.
+  const bool all_first = kv->upload_by_kernel;
+  for (int c = 0; c < (all_first ? n_chunks : 1); ++c)
+    if ((rc = copy_in(c)) != TIDE_OK) return rc;
+  int64_t launches = 0, dec_items = 0, pre_items = 0, mrg_rows = 0;
+  std::vector<int32_t> ip;
+  for (int c = 0; c < n_chunks; ++c) {
+    const int r0 = cut[c], r1 = cut[c + 1];
+    const size_t t0 = (size_t)indptr[(size_t)r0], tn = (size_t)indptr[(size_t)r1] - t0;
+    cudaEvent_t ev_done = kv->ev_host[kMaxHostChunks + c];
+    if (n_chunks > 1 && cudaStreamWaitEvent(st, kv->ev_host[c], 0) != cudaSuccess) return TIDE_ERR_CUDA;
+    ip.assign((size_t)(r1 - r0) + 1, 0);
+    for (int b = r0; b <= r1; ++b) ip[(size_t)(b - r0)] = indptr[(size_t)b] - (int32_t)t0;
+    rc = tide_kv_append(kv, layer, r1 - r0, ids.data() + r0, ip.data(), dk + t0 * kv_row, dv + t0 * kv_row, stream);
+    if (rc != TIDE_OK) return rc;
+    rc = tide_attend(kv, layer, r1 - r0, rows + r0, nullptr, dq + t0 * q_row, scale, dout + t0 * q_row,
+                     lse ? dlse + t0 * g.Hq : nullptr, stream);
+    if (rc != TIDE_OK) return rc;
+    launches += kv->last_launches; dec_items += kv->last_decode_items; pre_items += kv->last_prefill_items; mrg_rows += kv->last_merge_rows;
+    if (!all_first && c + 1 < n_chunks && (rc = copy_in(c + 1)) != TIDE_OK) return rc;
+    if (n_chunks > 1 && (cudaEventRecord(ev_done, st) != cudaSuccess || cudaStreamWaitEvent(s_out, ev_done, 0) != cudaSuccess))
+      return TIDE_ERR_CUDA;
+    if (cudaMemcpyAsync((uint8_t*)out + t0 * q_row, dout + t0 * q_row, tn * q_row, cudaMemcpyDeviceToHost, s_out) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (lse && cudaMemcpyAsync(lse + t0 * g.Hq, dlse + t0 * g.Hq, tn * lse_row, cudaMemcpyDeviceToHost, s_out) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
+  kv->last_launches = launches; kv->last_decode_items = dec_items; kv->last_prefill_items = pre_items; kv->last_merge_rows = mrg_rows;
+  if (n_chunks > 1) {
+    // the caller's stream ends after the last copy out, so stream order still means "the step is complete"
+    if (cudaEventRecord(ev_end, s_out) != cudaSuccess || cudaStreamWaitEvent(st, ev_end, 0) != cudaSuccess) return TIDE_ERR_CUDA;
+  }
   if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
   return TIDE_OK;
 }

@@ -93,6 +93,7 @@ struct AppendParams {
 };
 
 cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s);
+cudaError_t launch_upload(void* dst, const void* src_mapped_host, size_t bytes, cudaStream_t s);   // bytes % 4 == 0
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s);
 cudaError_t launch_copy_pages(uint8_t* pool, const int32_t* src, const int32_t* dst, int n, long long page_bytes, cudaStream_t s);
 cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int pos0, int len, uint16_t* out_k,

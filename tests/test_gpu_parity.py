@@ -210,8 +210,12 @@ def test_append_leaves_neighbouring_slots_untouched(env):
     kv.close()
 
 
-def test_step_host_matches_append_then_attend(env):
+@pytest.mark.parametrize("groups", [0, 3, 8])
+def test_step_host_matches_append_then_attend(env, groups, monkeypatch):
+    # groups > 0 forces the step to be cut into that many row groups whose copies and kernels overlap (what large
+    # steps do by themselves); pages, cache bits and outputs must not depend on the cut
     tide, torch = env
+    monkeypatch.setenv("TIDE_HOST_STEP_CHUNKS", str(groups))
     w = inputs.make_workload(1)
     kv_bits = [w.task_kv(b) for b in range(w.B)]
     q_bits = np.concatenate([w.task_q(b) for b in range(w.B)])
@@ -229,6 +233,7 @@ def test_step_host_matches_append_then_attend(env):
     hout = torch.zeros((total_q, w.Hq, w.D), dtype=torch.int16).pin_memory()
     hlse = torch.zeros((total_q, w.Hq), dtype=torch.float32).pin_memory()
     kv.step_host(w.rows(), hk, hv, hq, w.scale, hout, hlse)
+    assert kv.status() == tide.OK
     H.compare_bookkeeping(w, c, kv)
     H.compare_cache(w, c, kv)
     ref_o, ref_l = H.oracle_attend(c, w, q_bits)
