@@ -112,6 +112,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
   for (int i = 0; i < 32; ++i) u[i] = __float_as_uint(v[i]);
   tmem_st32u(taddr, u);
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -382,20 +387,23 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 #pragma unroll
         for (int c = 0; c < 64; ++c) if (c >= vis) s[c] = -INFINITY;
       }
-      // independent partial reductions: one long dependent chain would expose its latency
+      // independent partial reductions (one long dependent chain would expose its latency), three inputs per
+      // instruction: 8 chains of 4 over 64 values, then a tree
       float mxp[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(s[i], s[i + 8]);
+      for (int i = 0; i < 8; ++i) mxp[i] = max3(s[i], s[i + 8], s[i + 16]);
 #pragma unroll
-      for (int c = 16; c < 64; c += 16) {
+      for (int i = 0; i < 8; ++i) mxp[i] = max3(mxp[i], s[i + 24], s[i + 32]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(mxp[i], fmaxf(s[c + i], s[c + i + 8]));
-      }
-      float mx = fmaxf(fmaxf(fmaxf(mxp[0], mxp[1]), fmaxf(mxp[2], mxp[3])), fmaxf(fmaxf(mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7])));
+      for (int i = 0; i < 8; ++i) mxp[i] = max3(mxp[i], s[i + 40], s[i + 48]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(mxp[i], s[i + 56]);
+      float mx = max3(max3(mxp[0], mxp[1], mxp[2]), max3(mxp[3], mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7]));
       mx *= sl2;                                               // scale > 0 on this path
       float m_new = m;
       if (mx > m + kRescaleThreshold || m == -INFINITY) m_new = fmaxf(m, mx);
-      const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);   // m = -inf -> 0
+      float alpha = 1.f;
+      if (__any_sync(0xffffffffu, m_new != m)) alpha = fast_exp2(m - m_new);   // rare; m = -inf -> 0, equal -> 1
       if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         // O_t holds tiles < j: S_t(j) was committed after PV_t(j-1)
 #pragma unroll
