@@ -133,7 +133,17 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
     atomicAdd(c + (i1), (unsigned long long)tt_wait2);                                              \
     atomicAdd(c + (i2), (unsigned long long)(clock64() - tt_t0));                                   \
   } while (0)
+// per-phase accounting: TT_PH(i) adds the cycles since the previous mark to phase i
+#define TT_PH_DECL long long tt_ph[6] = {0, 0, 0, 0, 0, 0}, tt_b = 0
+#define TT_PH_START tt_b = clock64()
+#define TT_PH(i) do { const long long now_ = clock64(); tt_ph[i] += now_ - tt_b; tt_b = now_; } while (0)
+#define TT_PH_FLUSH(i0) do { unsigned long long* c = reinterpret_cast<unsigned long long*>(P.status) + 8; \
+    for (int i_ = 0; i_ < 6; ++i_) atomicAdd(c + (i0) + i_, (unsigned long long)tt_ph[i_]); } while (0)
 #else
+#define TT_PH_DECL
+#define TT_PH_START
+#define TT_PH(i)
+#define TT_PH_FLUSH(i0)
 #define TT_DECL
 #define TT_BEGIN
 #define TT_END(acc)
@@ -270,6 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       // ================= MMA issuer (whole warp converged, one elected lane issues) =================
       if (n_tiles > 0) {
         TT_DECL;
+        TT_PH_DECL;
         mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
         tc_fence_after();
         auto issue_qk = [&](int t, int j) {
@@ -309,22 +320,29 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
             __syncwarp();
           }
           bool k_ready = false;
+          TT_PH_START;
           for (int t = 0; t < 2; ++t) {
             if (j < t_tiles[t]) {
               TT_BEGIN;
               mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
               TT_END(tt_wait);
+              TT_PH(0);
               tc_fence_after();
+              TT_PH(1);
               issue_pv(t, j);
+              TT_PH(2);
               if (j + 1 < t_tiles[t]) {
                 if (!k_ready) { wait_full(j + 1); k_ready = true; }
+                TT_PH(3);
                 issue_qk(t, j + 1);                          // overwrites S_t / P_t after PV_t(j), in order
+                TT_PH(4);
               } else {
                 mma_commit(smem_u32(&bars.o_full[t]));
               }
             }
           }
           mma_commit(smem_u32(&bars.kv_empty[j % kNumBuf]));   // K_j and V_j are consumed once PV(j) retires
+          TT_PH(5);
         }
         // every MMA has completed (commits arrive in issue order) before this thread leaves
         {
@@ -332,7 +350,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
         }
 #ifdef TIDE_UMMA_TIMING
-        if (lane == 0) TT_FLUSH(2, 3, 4);
+        if (lane == 0) { TT_FLUSH(2, 3, 4); TT_PH_FLUSH(12); }   // counters 12..17: wait P, fence, PV, wait K/V, QK, commits
 #endif
       }
     }
@@ -372,15 +390,18 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const uint32_t o_addr = tmem + lane_addr + kColO + t * 128;
 
     TT_DECL;
+    TT_PH_DECL;
     for (int j = 0; j < my_tiles; ++j) {
       TT_BEGIN;
       mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
       TT_END(tt_wait);
+      TT_PH_START;
       tc_fence_after();
       float s[64];
       tmem_ld32(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
       tmem_ld32(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_wait_ld();
+      TT_PH(0);
       const int tile_key0 = kv_begin + j * kTileKeys;
       if (tile_key0 + kTileKeys > t_min_limit[t]) {            // uniform over the warpgroup
         const int vis = limit - tile_key0;
@@ -417,6 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
         }
       }
       m = m_new;
+      TT_PH(1);
       const float mu = (m == -INFINITY) ? 0.f : m;
       float sp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
@@ -431,11 +453,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 #pragma unroll
         for (int i = 0; i < 4; ++i) pk[(c >> 1) + i] = pack_bf16(s[c + 2 * i], s[c + 2 * i + 1]);
       }
+      TT_PH(2);
       tmem_st32u(s_addr, pk);                                  // P_t over the first 32 columns of S_t
       l = l * alpha + (((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7])));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&bars.p_full[t]));
+      TT_PH(3);
     }
 
     // ---- epilogue: O / l and LSE ----
@@ -447,7 +471,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       tc_fence_after();
     }
 #ifdef TIDE_UMMA_TIMING
-    if (lane == 0 && (warp & 3) == 0) TT_FLUSH(0, 1, 5);
+    if (lane == 0 && (warp & 3) == 0) { TT_FLUSH(0, 1, 5); TT_PH_FLUSH(6); }   // counters 6..9: load, max, exp, store
 #endif
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const float e2 = l > 0.f ? m + log2f(l) : -INFINITY;
