@@ -231,7 +231,7 @@ int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile
  * global mode, where cudaMalloc is refused; processes whose framework allocator already owns the whole device,
  * so a fresh cudaMalloc fails; and steps that cannot afford the device-wide synchronisation cudaMalloc implies.
  * Same semantics, arguments and results as tide_attend restricted to such rows, with the library's own page
- * table.  Limits: at most TIDE_STATIC_MAX_ROWS rows per call (more returns TIDE_ERR_WORKSPACE), decode-style
+ * table, on layer 0.  Limits: at most TIDE_STATIC_MAX_ROWS rows per call (more returns TIDE_ERR_WORKSPACE), decode-style
  * rows only (others return TIDE_ERR_INVALID_ARG); long rows are split over KV only as far as the fixed array
  * allows.  The first call on a device looks up the array's device address; make that call before any stream
  * capture begins.  Every call uses the same array and overwrites what the previous call left there (nothing in

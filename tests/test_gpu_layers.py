@@ -287,3 +287,48 @@ def test_layers_of_a_step_replayed_from_a_cuda_graph():
     _same_state(kv, orc, tasks)
     _same_bits(kv, orc, tasks, L)
     kv.close()
+
+
+def test_layer_pools_beyond_four_gib():
+    """Three layers of 2.46 GB each, with the tasks' pages at the far end of every layer's pool: byte offsets of
+    layers 1 and 2 lie beyond 4 GiB, so any 32-bit step in the address arithmetic would show."""
+    import torch
+    from paper_2608_10402_b200 import tide
+    HQ, HKV, D, S, L = 28, 4, 128, 16, 3
+    NUM_PAGES, USED = 150000, 64
+    free, _ = torch.cuda.mem_get_info()
+    if free < 10 * (1 << 30):
+        pytest.skip("needs 10 GB of free device memory")
+    rng = np.random.default_rng(10)
+    scale = 1.0 / math.sqrt(D)
+    # the library hands out the last USED pages first; the oracle runs on a pool of just those pages
+    order = np.concatenate([np.arange(NUM_PAGES - USED, NUM_PAGES), np.arange(NUM_PAGES - USED)]).astype(np.int32)
+    kv = tide.TideKV(HQ, HKV, D, S, NUM_PAGES, 4, 64, 4, 1024, free_order=order, num_layers=L)
+    orc = LayeredKVOracle(L, num_pages=USED, page_size=S, num_kv_heads=HKV, head_dim=D, max_tasks=4, max_pages_per_task=64)
+    tasks = [0, 1, 2]
+    for t in tasks:
+        kv.alloc(t)
+        orc.alloc(t)
+    cnt = [300, 17, 150]
+    for step_cnt in (cnt, [1, 40, 200]):
+        indptr = np.concatenate([[0], np.cumsum(step_cnt)]).astype(np.int32)
+        T = int(indptr[-1])
+        nk = np.stack([inputs.normal_bf16(rng, (T, HKV, D)) for _ in range(L)])
+        nv = np.stack([inputs.normal_bf16(rng, (T, HKV, D)) for _ in range(L)])
+        q = np.stack([inputs.normal_bf16(rng, (T, HQ, D)) for _ in range(L)])
+        orc.append(tasks, indptr, nk, nv)
+        rows = [(t, c, orc.task_len(t)) for t, c in zip(tasks, step_cnt)]
+        out = torch.zeros((L, T, HQ, D), dtype=torch.int16, device="cuda")
+        lse = torch.zeros((L, T, HQ), dtype=torch.float32, device="cuda")
+        dk, dv, dq = H.to_dev(nk, torch), H.to_dev(nv, torch), H.to_dev(q, torch)
+        kv.step_begin(rows)
+        for l in range(L):
+            kv.step_layer(l, dk[l], dv[l], dq[l], scale, out[l], lse[l])
+        assert kv.status() == tide.OK
+        for l in range(L):
+            ref_o, ref_l = cbuild.attend_paged(orc.layer(l), rows, q[l], scale)
+            H.check_outputs(H.from_dev(out[l]), lse[l].cpu().numpy(), ref_o, ref_l, f"layer {l}")
+    for t in tasks:
+        assert np.array_equal(kv.page_table(t), orc.page_table(t) + (NUM_PAGES - USED))
+    _same_bits(kv, orc, tasks, L)
+    kv.close()
