@@ -205,6 +205,39 @@ def multi_layer_leg(args, w, torch, tide, seed):
                 stream.synchronize()
             res[name] = {"device_ms_per_layer": e0.elapsed_time(e1) / args.steps / L,
                          "host_enqueue_ms_per_step": float(np.median(host))}
+        # the same with launch shapes fixed at twice what this step plans: ONE graph then serves every later step
+        # whose plan stays below those maxima (surplus thread blocks leave at once)
+        kv.step_begin(rows, stream=stream)
+        pl = kv.last_plan()
+        rollback()
+        n_dec = sum(1 for (_, n, _) in w.rows() if n * (w.Hq // w.Hkv) <= 16)
+        kv.step_fix_grids(max_decode_items=2 * pl["decode_items"] + 64,
+                          max_tile_items=0 if w.D == 128 else 2 * pl["prefill_items"] + 64,
+                          max_umma_items=2 * pl["prefill_items"] + 64 if w.D == 128 and n_dec < w.B else 0,
+                          max_merge_rows=min(2 * pl["merge_rows"] + 64, total_q * w.Hq), max_tokens=total_q)
+        kv.step_begin(rows, stream=stream)
+        graph2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph2, stream=stream):
+            for l in range(L):
+                kv.step_layer(l, new_k[l], new_v[l], q[l], w.scale, out[l], lse[l], stream=torch.cuda.current_stream())
+        rollback()
+
+        def from_fixed_graph():
+            kv.step_begin(rows, stream=stream)
+            graph2.replay()
+
+        for _ in range(3):
+            from_fixed_graph()
+            rollback()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            from_fixed_graph()
+            rollback()
+        e1.record(stream)
+        stream.synchronize()
+        res["graph_fixed_shapes"] = {"device_ms_per_layer": e0.elapsed_time(e1) / args.steps / L}
         assert kv.status(stream=stream) == tide.OK
     kv.close()
     return {"layers": L, "graph_capture_ms": capture_ms, **res}

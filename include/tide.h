@@ -157,6 +157,15 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
  * as the captured pointers stay valid.  scale must be positive and finite.  TIDE_ERR_INVALID_ARG if no step is
  * open.  Per-phase timing (tide_set_profiling) does not cover tide_step_layer. */
 int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows /*host*/, void* stream);
+/* Fixes the launch shapes of tide_step_layer so that ONE captured CUDA graph of a step's layers can be replayed
+ * for later steps with other rows: every kernel is launched with a grid sized for the given maxima (work items of
+ * the decode-style, warp-MMA tile and tcgen05 kernels, rows of the merge, new tokens) and reads the step's real
+ * counts from the step area that tide_step_begin fills; surplus thread blocks leave at once.  A maximum of 0
+ * means that kind of launch is left out.  tide_step_begin refuses a step that plans more than a maximum with
+ * TIDE_ERR_WORKSPACE (tide_last_plan shows what a step planned).  All five 0 turns the mode off (the default:
+ * exact grids).  Closes an open step.  max_tokens may not exceed max_batch_tokens. */
+int tide_step_fix_grids(tide_kv_t* kv, int32_t max_decode_items, int32_t max_tile_items, int32_t max_umma_items,
+                        int32_t max_merge_rows, int32_t max_tokens);
 int tide_step_layer(tide_kv_t* kv, int32_t layer, const void* new_k /*device*/, const void* new_v /*device*/,
                     const void* q /*device*/, float scale, void* out /*device*/, float* lse /*device or NULL*/,
                     void* stream);

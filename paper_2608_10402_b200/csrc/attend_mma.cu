@@ -53,7 +53,12 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
 
   // ---- which item ----
   const int item = blockIdx.x;
-  const int si = find_segment(P.n_segs, item, [&](int i) { return P.segs[i].item_base; });
+  int n_segs = P.n_segs;
+  if (P.dyn != nullptr) {                      // fixed grid: the batch's counts live in device memory
+    if (item >= P.dyn[0]) return;
+    n_segs = P.dyn[1];
+  }
+  const int si = find_segment(n_segs, item, [&](int i) { return P.segs[i].item_base; });
   const Segment seg = P.segs[si];
   int local = item - seg.item_base;
   const int m_tile = local % seg.n_mtiles;
@@ -390,16 +395,18 @@ cudaError_t attend_kernels_init() {
 }
 
 cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s) {
-  if (p.n_items <= 0) return cudaSuccess;
-  if (p.g.D == 128) attend_mma_kernel<128, true><<<p.n_items, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
-  else attend_mma_kernel<64, true><<<p.n_items, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
+  const int grid = p.dyn ? p.grid_cap : p.n_items;
+  if (grid <= 0) return cudaSuccess;
+  if (p.g.D == 128) attend_mma_kernel<128, true><<<grid, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
+  else attend_mma_kernel<64, true><<<grid, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
   return cudaGetLastError();
 }
 
 cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s) {
-  if (p.n_items <= 0) return cudaSuccess;
-  if (p.g.D == 128) attend_mma_kernel<128, false><<<p.n_items, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
-  else attend_mma_kernel<64, false><<<p.n_items, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
+  const int grid = p.dyn ? p.grid_cap : p.n_items;
+  if (grid <= 0) return cudaSuccess;
+  if (p.g.D == 128) attend_mma_kernel<128, false><<<grid, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(p);
+  else attend_mma_kernel<64, false><<<grid, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -409,8 +416,9 @@ cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s) {
 __global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
   const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  if (row >= P.n_rows) return;
-  const int si = find_segment(P.n_segs, row, [&](int i) { return P.segs[i].merge_base; });
+  const int n_rows = P.dyn ? P.dyn[0] : P.n_rows, n_segs = P.dyn ? P.dyn[1] : P.n_segs;
+  if (row >= n_rows) return;
+  const int si = find_segment(n_segs, row, [&](int i) { return P.segs[i].merge_base; });
   const Segment seg = P.segs[si];
   const int local = row - seg.merge_base;                 // token * Hq + head inside the segment
   const long long stride = (long long)seg.n * P.Hq;       // partial rows per split
@@ -450,8 +458,9 @@ __global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
 }
 
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t s) {
-  if (p.n_rows <= 0) return cudaSuccess;
-  const int blocks = (p.n_rows + 7) / 8;
+  const int rows = p.dyn ? p.grid_cap_rows : p.n_rows;
+  if (rows <= 0) return cudaSuccess;
+  const int blocks = (rows + 7) / 8;
   merge_kernel<<<blocks, 256, 0, s>>>(p);
   return cudaGetLastError();
 }

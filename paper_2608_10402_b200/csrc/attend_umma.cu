@@ -172,7 +172,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 
   // ---- which item ----
   const int item = blockIdx.x;
-  const int si = find_segment(P.n_segs, item, [&](int i) { return P.segs[i].item_base; });
+  int n_segs = P.n_segs;
+  if (P.dyn != nullptr) {                      // fixed grid: the batch's counts live in device memory
+    if (item >= P.dyn[0]) return;
+    n_segs = P.dyn[1];
+  }
+  const int si = find_segment(n_segs, item, [&](int i) { return P.segs[i].item_base; });
   const Segment seg = P.segs[si];
   int local = item - seg.item_base;
   const int m_tile = local % seg.n_mtiles;
@@ -527,8 +532,9 @@ cudaError_t attend_umma_init() {
 }
 
 cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s) {
-  if (p.n_items <= 0) return cudaSuccess;
-  umma::attend_umma_kernel<<<p.n_items, umma::kThreads, umma::kSmemBytes, s>>>(p);
+  const int grid = p.dyn ? p.grid_cap : p.n_items;
+  if (grid <= 0) return cudaSuccess;
+  umma::attend_umma_kernel<<<grid, umma::kThreads, umma::kSmemBytes, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -51,7 +51,8 @@ constexpr int kAppendMaxRecsSmem = 1024;
 // per-chunk index split needs no division.
 __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const AppendParams P) {
   __shared__ int32_t s_tok0[kAppendMaxRecsSmem];
-  const int n_recs = P.n_recs;
+  const int n_recs = P.dyn ? P.dyn[0] : P.n_recs;
+  const int n_tokens = P.dyn ? P.dyn[1] : P.n_tokens;
   const bool in_smem = n_recs <= kAppendMaxRecsSmem;
   if (in_smem) {
     for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = P.recs[i].tok0;
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const Ap
   const int rows2 = 2 * P.g.Hkv;              // K rows then V rows of one token
   const int cpt = rows2 * cpr;                // chunks per token
   const int warps_total = gridDim.x * (kAppendThreads / 32);
-  for (int tok = blockIdx.x * (kAppendThreads / 32) + (threadIdx.x >> 5); tok < P.n_tokens; tok += warps_total) {
+  for (int tok = blockIdx.x * (kAppendThreads / 32) + (threadIdx.x >> 5); tok < n_tokens; tok += warps_total) {
     int r;
     if (in_smem) r = find_segment(n_recs, tok, [&](int i) { return s_tok0[i]; });
     else r = find_segment(n_recs, tok, [&](int i) { return P.recs[i].tok0; });
@@ -89,8 +90,9 @@ __global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const Ap
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
-  if (p.n_tokens <= 0) return cudaSuccess;
-  long long blocks = ((long long)p.n_tokens + kAppendThreads / 32 - 1) / (kAppendThreads / 32);
+  const int tokens = p.dyn ? p.grid_cap_tokens : p.n_tokens;
+  if (tokens <= 0) return cudaSuccess;
+  long long blocks = ((long long)tokens + kAppendThreads / 32 - 1) / (kAppendThreads / 32);
   const long long cap = 148LL * 8 * 8;   // 8 resident blocks per SM, a few tokens per warp beyond this
   if (blocks > cap) blocks = cap;
   append_scatter_kernel<<<(unsigned)blocks, kAppendThreads, 0, s>>>(p);

@@ -24,6 +24,8 @@ constexpr int kSlotRecs = 2048;              // most append records per upload
 constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
 constexpr int kNumSms = 148;
 constexpr long long kPartRowsBase = 256 * 1024;
+// header of the step area (int32 words): counts a fixed-shape launch reads on the device, as (count, segments) pairs
+constexpr int kHdrRecs = 0, kHdrDecItems = 2, kHdrTileItems = 4, kHdrUmmaItems = 6, kHdrMergeRows = 8;
 constexpr int kMaxHostChunks = 8;                 // most row groups of one host-buffer step
 constexpr size_t kHostChunkBytes = 64u << 20;      // transfer bytes per group from which cutting a step pays
 
@@ -41,7 +43,7 @@ struct Layout {
 // A planned batch as the launches need it: where the four segment arrays sit on the device and how many work
 // items each launch has.
 struct PlanDev {
-  const Segment* segs = nullptr;   // [decode][tile][tcgen05][merge]
+  const Segment *seg_dec = nullptr, *seg_tile = nullptr, *seg_umma = nullptr, *seg_merge = nullptr;
   size_t n_dec = 0, n_tile = 0, n_umma = 0, n_merge = 0;
   long long items_dec = 0, items_tile = 0, items_umma = 0, merge_rows = 0;
 };
@@ -103,6 +105,9 @@ struct tide_kv {
   bool step_upload_pending = false, step_valid = false;
   PlanDev step_plan;
   int step_recs = 0, step_tokens = 0;
+  // fixed launch shapes for tide_step_layer (0 = off): most work items / rows / tokens a step may plan
+  bool fixed_grids = false;
+  int cap_dec = 0, cap_tile = 0, cap_umma = 0, cap_merge_rows = 0, cap_tokens = 0;
   // host-buffer steps: copy streams and the events that order them against the caller's stream
   cudaStream_t st_in = nullptr, st_out = nullptr;
   cudaEvent_t ev_host[2 * kMaxHostChunks + 2] = {};   // copies-in done, kernels done (per group); start, end
@@ -144,8 +149,9 @@ Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
   L.off_status = off; off += 256;
   L.off_table = off; off = align_up(off + (size_t)c->max_tasks * c->max_pages_per_task * 4, 256);
   L.off_old_row = off; off = align_up(off + (size_t)c->max_pages_per_task * 4 + 64, 256);   // row + one page pair
-  L.step_seg_off = align_up((size_t)c->max_batch_rows * sizeof(AppendRec), 256);
-  L.step_bytes = align_up(L.step_seg_off + (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
+  // step area: 256-byte header of counts | write records | four segment arrays of max_batch_rows entries each
+  L.step_seg_off = align_up(256 + (size_t)c->max_batch_rows * sizeof(AppendRec), 256);
+  L.step_bytes = align_up(L.step_seg_off + (size_t)(4 * c->max_batch_rows) * sizeof(Segment), 256);
   L.off_step = off; off += L.step_bytes;
   L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 + (size_t)kSlotRecs * 8 +
                               (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
@@ -900,15 +906,18 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
   return TIDE_OK;
 }
 
-// Writes the four segment arrays one after the other at `h` and describes them as they will sit at `d`.
-static PlanDev pack_plan(const PlanHost& P, Segment* h, const Segment* d) {
-  Segment* w = h;
-  w = std::copy(P.seg_dec.begin(), P.seg_dec.end(), w);
-  w = std::copy(P.seg_tile.begin(), P.seg_tile.end(), w);
-  w = std::copy(P.seg_umma.begin(), P.seg_umma.end(), w);
-  std::copy(P.seg_merge.begin(), P.seg_merge.end(), w);
+// Writes the four segment arrays at `h` and describes them as they will sit at `d`: one after the other
+// (stride 0), or each at a fixed distance of `stride` entries, so that their addresses do not depend on the batch.
+static PlanDev pack_plan(const PlanHost& P, Segment* h, const Segment* d, size_t stride) {
+  const size_t o_tile = stride ? stride : P.seg_dec.size();
+  const size_t o_umma = stride ? 2 * stride : o_tile + P.seg_tile.size();
+  const size_t o_merge = stride ? 3 * stride : o_umma + P.seg_umma.size();
+  std::copy(P.seg_dec.begin(), P.seg_dec.end(), h);
+  std::copy(P.seg_tile.begin(), P.seg_tile.end(), h + o_tile);
+  std::copy(P.seg_umma.begin(), P.seg_umma.end(), h + o_umma);
+  std::copy(P.seg_merge.begin(), P.seg_merge.end(), h + o_merge);
   PlanDev pd;
-  pd.segs = d;
+  pd.seg_dec = d; pd.seg_tile = d + o_tile; pd.seg_umma = d + o_umma; pd.seg_merge = d + o_merge;
   pd.n_dec = P.seg_dec.size(); pd.n_tile = P.seg_tile.size(); pd.n_umma = P.seg_umma.size(); pd.n_merge = P.seg_merge.size();
   pd.items_dec = P.items_dec; pd.items_tile = P.items_tile; pd.items_umma = P.items_umma; pd.merge_rows = P.merge_rows;
   return pd;
@@ -917,7 +926,7 @@ static PlanDev pack_plan(const PlanHost& P, Segment* h, const Segment* d) {
 // The attention launches of one planned batch on one layer: kernel launches only (and, with `events`, the phase
 // time stamps), so a caller may capture them in a CUDA graph.
 static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32_t* page_table, const void* q, float scale,
-                       void* out, float* lse, cudaStream_t st, bool events, int64_t* n_launches) {
+                       void* out, float* lse, cudaStream_t st, bool events, int64_t* n_launches, const int32_t* dyn) {
   AttendParams ap;
   ap.pool = kv->layer_pool(layer);
   ap.table = page_table ? page_table : kv->d_table;
@@ -930,31 +939,36 @@ static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32
   ap.status = kv->d_status;
   ap.g = kv->g;
   int64_t launches = 0;
+  // dyn != nullptr: fixed launch shapes; the counts of the batch are read on the device (header of the step area)
   if (events) cudaEventRecord(kv->ev_attend[0], st);
-  if (d.items_dec > 0) {
-    ap.segs = d.segs; ap.n_segs = (int)d.n_dec; ap.n_items = (int)d.items_dec;
+  if (dyn ? kv->cap_dec > 0 : d.items_dec > 0) {
+    ap.segs = d.seg_dec; ap.n_segs = (int)d.n_dec; ap.n_items = (int)d.items_dec;
+    ap.dyn = dyn ? dyn + kHdrDecItems : nullptr; ap.grid_cap = kv->cap_dec;
     if (launch_attend_decode(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
   if (events) cudaEventRecord(kv->ev_attend[1], st);
-  if (d.items_tile > 0) {
-    ap.segs = d.segs + d.n_dec; ap.n_segs = (int)d.n_tile; ap.n_items = (int)d.items_tile;
+  if (dyn ? kv->cap_tile > 0 : d.items_tile > 0) {
+    ap.segs = d.seg_tile; ap.n_segs = (int)d.n_tile; ap.n_items = (int)d.items_tile;
+    ap.dyn = dyn ? dyn + kHdrTileItems : nullptr; ap.grid_cap = kv->cap_tile;
     if (launch_attend_tile(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
-  if (d.items_umma > 0) {
-    ap.segs = d.segs + d.n_dec + d.n_tile; ap.n_segs = (int)d.n_umma; ap.n_items = (int)d.items_umma;
+  if (dyn ? kv->cap_umma > 0 : d.items_umma > 0) {
+    ap.segs = d.seg_umma; ap.n_segs = (int)d.n_umma; ap.n_items = (int)d.items_umma;
+    ap.dyn = dyn ? dyn + kHdrUmmaItems : nullptr; ap.grid_cap = kv->cap_umma;
     if (launch_attend_umma(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
   if (events) cudaEventRecord(kv->ev_attend[2], st);
-  if (d.merge_rows > 0) {
+  if (dyn ? kv->cap_merge_rows > 0 : d.merge_rows > 0) {
     MergeParams mp;
-    mp.segs = d.segs + d.n_dec + d.n_tile + d.n_umma;
+    mp.segs = d.seg_merge;
     mp.n_segs = (int)d.n_merge;
     mp.n_rows = (int)d.merge_rows;
     mp.part_o = kv->d_part_o; mp.part_lse = kv->d_part_lse;
     mp.out = (uint16_t*)out; mp.lse = lse; mp.Hq = kv->g.Hq; mp.D = kv->g.D;
+    mp.dyn = dyn ? dyn + kHdrMergeRows : nullptr; mp.grid_cap_rows = kv->cap_merge_rows;
     if (launch_merge(mp, st) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
@@ -982,17 +996,29 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   cudaStream_t st = (cudaStream_t)stream;
   Slot* slot;
   if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
-  const PlanDev pd = pack_plan(P, (Segment*)(slot->host + 256), (const Segment*)(slot->dev + 256));
+  const PlanDev pd = pack_plan(P, (Segment*)(slot->host + 256), (const Segment*)(slot->dev + 256), 0);
   if (upload(kv, slot->dev + 256, slot->host + 256, P.n_all() * sizeof(Segment), st) != cudaSuccess)
     return TIDE_ERR_CUDA;
   int64_t launches = 0;
-  if ((rc = launch_plan(kv, layer, pd, page_table, q, scale, out, lse, st, kv->profiling, &launches)) != TIDE_OK) return rc;
+  if ((rc = launch_plan(kv, layer, pd, page_table, q, scale, out, lse, st, kv->profiling, &launches, nullptr)) != TIDE_OK) return rc;
   if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   kv->last_decode_items = pd.items_dec;
   kv->last_prefill_items = pd.items_tile + pd.items_umma;
   kv->last_merge_rows = pd.merge_rows;
   kv->last_launches = launches + kv->append_launches;
   kv->append_launches = 0;
+  return TIDE_OK;
+}
+
+int tide_step_fix_grids(tide_kv_t* kv, int32_t max_decode_items, int32_t max_tile_items, int32_t max_umma_items,
+                        int32_t max_merge_rows, int32_t max_tokens) {
+  if (kv == nullptr || max_decode_items < 0 || max_tile_items < 0 || max_umma_items < 0 || max_merge_rows < 0 || max_tokens < 0)
+    return TIDE_ERR_INVALID_ARG;
+  if (max_tokens > kv->cfg.max_batch_tokens) return TIDE_ERR_WORKSPACE;
+  kv->fixed_grids = (max_decode_items | max_tile_items | max_umma_items | max_merge_rows | max_tokens) != 0;
+  kv->cap_dec = max_decode_items; kv->cap_tile = max_tile_items; kv->cap_umma = max_umma_items;
+  kv->cap_merge_rows = max_merge_rows; kv->cap_tokens = max_tokens;
+  kv->step_valid = false;
   return TIDE_OK;
 }
 
@@ -1020,13 +1046,21 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
   // (and can still be refused) before anything changes.
   PlanHost P;
   if ((rc = build_plan(kv, n_rows, rows, g.D == 128, P)) != TIDE_OK) return rc;
-  if (kv->lay.step_seg_off + P.n_all() * sizeof(Segment) > kv->lay.step_bytes) return TIDE_ERR_WORKSPACE;
+  if (kv->fixed_grids && (P.items_dec > kv->cap_dec || P.items_tile > kv->cap_tile || P.items_umma > kv->cap_umma ||
+                          P.merge_rows > kv->cap_merge_rows || indptr[(size_t)n_rows] > kv->cap_tokens))
+    return TIDE_ERR_WORKSPACE;   // the step does not fit the launch shapes that were fixed
   cudaStream_t st = (cudaStream_t)stream;
   kv->append_launches = 0;
   if ((rc = extend_tasks(kv, n_rows, ids.data(), indptr.data(), st, nullptr)) != TIDE_OK) return rc;
   // one upload: the write records of the rows, then the segments
   if (kv->step_upload_pending && cudaEventSynchronize(kv->ev_step) != cudaSuccess) return TIDE_ERR_CUDA;
-  AppendRec* recs = (AppendRec*)kv->h_step;
+  int32_t* hdr = (int32_t*)kv->h_step;
+  hdr[kHdrRecs] = n_rows; hdr[kHdrRecs + 1] = indptr[(size_t)n_rows];
+  hdr[kHdrDecItems] = (int32_t)P.items_dec; hdr[kHdrDecItems + 1] = (int32_t)P.seg_dec.size();
+  hdr[kHdrTileItems] = (int32_t)P.items_tile; hdr[kHdrTileItems + 1] = (int32_t)P.seg_tile.size();
+  hdr[kHdrUmmaItems] = (int32_t)P.items_umma; hdr[kHdrUmmaItems + 1] = (int32_t)P.seg_umma.size();
+  hdr[kHdrMergeRows] = (int32_t)P.merge_rows; hdr[kHdrMergeRows + 1] = (int32_t)P.seg_merge.size();
+  AppendRec* recs = (AppendRec*)(kv->h_step + 256);
   for (int b = 0; b < n_rows; ++b) {
     recs[b].table_off = rows[b].task * g.max_pages_per_task;
     recs[b].pos0 = rows[b].ctx_len - rows[b].q_len;
@@ -1034,9 +1068,18 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
     recs[b].count = rows[b].q_len;
   }
   uint8_t* d_step = kv->ws + kv->lay.off_step;
-  kv->step_plan = pack_plan(P, (Segment*)(kv->h_step + kv->lay.step_seg_off), (const Segment*)(d_step + kv->lay.step_seg_off));
-  if (cudaMemcpyAsync(d_step, kv->h_step, kv->lay.step_seg_off + P.n_all() * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess)
+  const size_t stride = (size_t)kv->cfg.max_batch_rows;
+  kv->step_plan = pack_plan(P, (Segment*)(kv->h_step + kv->lay.step_seg_off), (const Segment*)(d_step + kv->lay.step_seg_off), stride);
+  // header and records in one copy, then each segment array that is not empty (their places are fixed)
+  if (cudaMemcpyAsync(d_step, kv->h_step, 256 + (size_t)n_rows * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return TIDE_ERR_CUDA;
+  const size_t counts[4] = {P.seg_dec.size(), P.seg_tile.size(), P.seg_umma.size(), P.seg_merge.size()};
+  for (int a = 0; a < 4; ++a) {
+    const size_t off = kv->lay.step_seg_off + (size_t)a * stride * sizeof(Segment);
+    if (counts[a] > 0 &&
+        cudaMemcpyAsync(d_step + off, kv->h_step + off, counts[a] * sizeof(Segment), cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return TIDE_ERR_CUDA;
+  }
   if (cudaEventRecord(kv->ev_step, st) != cudaSuccess) return TIDE_ERR_CUDA;
   kv->step_upload_pending = true;
   kv->step_recs = n_rows;
@@ -1059,7 +1102,10 @@ int tide_step_layer(tide_kv_t* kv, int32_t layer, const void* new_k, const void*
   AppendParams ap;
   ap.pool = kv->layer_pool(layer);
   ap.table = kv->d_table;
-  ap.recs = (const AppendRec*)(kv->ws + kv->lay.off_step);
+  const int32_t* dyn = kv->fixed_grids ? (const int32_t*)(kv->ws + kv->lay.off_step) : nullptr;
+  ap.recs = (const AppendRec*)(kv->ws + kv->lay.off_step + 256);
+  ap.dyn = dyn ? dyn + kHdrRecs : nullptr;
+  ap.grid_cap_tokens = kv->cap_tokens;
   ap.n_recs = kv->step_recs;
   ap.n_tokens = kv->step_tokens;
   ap.new_k = (const uint16_t*)new_k;
@@ -1067,7 +1113,7 @@ int tide_step_layer(tide_kv_t* kv, int32_t layer, const void* new_k, const void*
   ap.g = kv->g;
   if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
   int64_t launches = 0;
-  const int rc = launch_plan(kv, layer, kv->step_plan, nullptr, q, scale, out, lse, st, false, &launches);
+  const int rc = launch_plan(kv, layer, kv->step_plan, nullptr, q, scale, out, lse, st, false, &launches, dyn);
   if (rc != TIDE_OK) return rc;
   kv->last_launches = launches + 1;
   return TIDE_OK;

@@ -61,6 +61,10 @@ struct AttendParams {
   float scale_log2e;
   int* status;
   Geom g;
+  // Fixed-grid mode (a launch that a CUDA graph replays for other batches): the launch has grid_cap CTAs and the
+  // kernel reads n_items = dyn[0] and n_segs = dyn[1] from device memory; CTAs beyond n_items leave at once.
+  const int32_t* dyn = nullptr;
+  int grid_cap = 0;
 };
 
 struct MergeParams {
@@ -72,6 +76,8 @@ struct MergeParams {
   uint16_t* out;
   float* lse;
   int Hq, D;
+  const int32_t* dyn = nullptr;   // fixed-grid mode: n_rows = dyn[0], n_segs = dyn[1]
+  int grid_cap_rows = 0;
 };
 
 struct __align__(16) AppendRec {
@@ -90,6 +96,8 @@ struct AppendParams {
   const uint16_t* new_k;
   const uint16_t* new_v;
   Geom g;
+  const int32_t* dyn = nullptr;   // fixed-grid mode: n_recs = dyn[0], n_tokens = dyn[1]
+  int grid_cap_tokens = 0;
 };
 
 cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s);

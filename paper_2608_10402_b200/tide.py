@@ -47,7 +47,7 @@ EXPORTS = [
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
     "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune", "tide_kv_fork", "tide_kv_page_refs",
-    "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer",
+    "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer", "tide_step_fix_grids",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -202,6 +202,11 @@ class TideKV:
     def step_begin(self, rows, stream=None):
         arr = rows if not isinstance(rows, (list, tuple)) else rows_array(rows)
         _check(lib.tide_step_begin(self.handle, ctypes.c_int32(len(arr)), arr, _stream(stream)), "tide_step_begin")
+
+    def step_fix_grids(self, max_decode_items=0, max_tile_items=0, max_umma_items=0, max_merge_rows=0, max_tokens=0):
+        _check(lib.tide_step_fix_grids(self.handle, ctypes.c_int32(max_decode_items), ctypes.c_int32(max_tile_items),
+                                       ctypes.c_int32(max_umma_items), ctypes.c_int32(max_merge_rows),
+                                       ctypes.c_int32(max_tokens)), "tide_step_fix_grids")
 
     def step_layer(self, layer, new_k, new_v, q, scale, out, lse=None, stream=None):
         _check(lib.tide_step_layer(self.handle, ctypes.c_int32(layer), _ptr(new_k), _ptr(new_v), _ptr(q),

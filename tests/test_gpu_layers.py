@@ -332,3 +332,75 @@ def test_layer_pools_beyond_four_gib():
         assert np.array_equal(kv.page_table(t), orc.page_table(t) + (NUM_PAGES - USED))
     _same_bits(kv, orc, tasks, L)
     kv.close()
+
+
+def test_one_graph_replayed_over_a_decode_loop():
+    """The generation loop between environment turns: the layers of a step are captured ONCE with fixed launch
+    shapes and replayed for every later step; only tide_step_begin (host planning, a small upload, the page-table
+    delta) runs between replays.  Lengths cross page boundaries, the KV splits change, and one step in the middle
+    also carries resume rows; every step is checked against the oracle."""
+    import torch
+    from paper_2608_10402_b200 import tide
+    HQ, HKV, D, S, L = 28, 4, 128, 16, 3
+    B, MAXQ = 6, 256
+    rng = np.random.default_rng(12)
+    scale = 1.0 / math.sqrt(D)
+    kv, orc = _make(L, HQ, HKV, D, S, 900, B, 128, B, MAXQ, rng)
+    tasks = list(range(B))
+    for t in tasks:
+        kv.alloc(t)
+        orc.alloc(t)
+    cnt = [int(rng.integers(60, 1500)) for _ in tasks]
+    indptr = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32)
+    T0 = int(indptr[-1])
+    hk = np.stack([inputs.normal_bf16(rng, (T0, HKV, D)) for _ in range(L)])
+    hv = np.stack([inputs.normal_bf16(rng, (T0, HKV, D)) for _ in range(L)])
+    orc.append(tasks, indptr, hk, hv)
+    kv.extend(tasks, indptr)
+    for l in range(L):
+        kv.write(l, tasks, indptr, H.to_dev(hk[l], torch), H.to_dev(hv[l], torch))
+    # static buffers the graph reads and writes; a step uses their first T rows
+    dk = torch.zeros((L, MAXQ, HKV, D), dtype=torch.int16, device="cuda")
+    dv = torch.zeros_like(dk)
+    dq = torch.zeros((L, MAXQ, HQ, D), dtype=torch.int16, device="cuda")
+    out = torch.zeros((L, MAXQ, HQ, D), dtype=torch.int16, device="cuda")
+    lse = torch.zeros((L, MAXQ, HQ), dtype=torch.float32, device="cuda")
+    kv.step_fix_grids(max_decode_items=1024, max_tile_items=64, max_umma_items=64, max_merge_rows=MAXQ * HQ, max_tokens=MAXQ)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = None
+    with torch.cuda.stream(side):
+        for step in range(24):
+            cnt = [1] * B if step != 9 else [1, 40, 1, 90, 1, 17]        # step 9 mixes in resume rows
+            indptr = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32)
+            T = int(indptr[-1])
+            nk = np.stack([inputs.normal_bf16(rng, (T, HKV, D)) for _ in range(L)])
+            nv = np.stack([inputs.normal_bf16(rng, (T, HKV, D)) for _ in range(L)])
+            q = np.stack([inputs.normal_bf16(rng, (T, HQ, D)) for _ in range(L)])
+            orc.append(tasks, indptr, nk, nv)
+            rows = [(t, c, orc.task_len(t)) for t, c in zip(tasks, cnt)]
+            dk[:, :T].copy_(H.to_dev(nk, torch))
+            dv[:, :T].copy_(H.to_dev(nv, torch))
+            dq[:, :T].copy_(H.to_dev(q, torch))
+            kv.step_begin(rows, stream=side)
+            if graph is None:
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for l in range(L):
+                        kv.step_layer(l, dk[l], dv[l], dq[l], scale, out[l], lse[l], stream=torch.cuda.current_stream())
+            graph.replay()
+            side.synchronize()
+            assert kv.status(stream=side) == tide.OK
+            for l in range(L):
+                ref_o, ref_l = cbuild.attend_paged(orc.layer(l), rows, q[l], scale)
+                H.check_outputs(H.from_dev(out[l, :T]), lse[l, :T].cpu().numpy(), ref_o, ref_l, f"step {step}, layer {l}")
+            _same_state(kv, orc, tasks)
+        # a step that plans more than the fixed shapes allow is refused before anything changes
+        kv.step_fix_grids(max_decode_items=2, max_tokens=MAXQ)
+        with pytest.raises(tide.TideError) as e:
+            kv.step_begin([(t, 1, orc.task_len(t) + 1) for t in tasks], stream=side)
+        assert e.value.code == tide.ERR_WORKSPACE
+        _same_state(kv, orc, tasks)
+    torch.cuda.current_stream().wait_stream(side)
+    _same_bits(kv, orc, tasks, L)
+    kv.close()
