@@ -70,3 +70,42 @@ def test_row_shapes_at_the_corners(geom):
     for t in ids:
         assert np.array_equal(kv.page_table(t), orc.page_table(t))
     kv.close()
+
+
+@pytest.mark.parametrize("scale", [0.0, -0.07])
+def test_non_positive_scale_takes_the_warp_mma_path(scale):
+    """The tcgen05 path takes the row maximum before scaling and so needs a positive scale; any other scale must
+    fall back to the warp-MMA tile path and still match the oracle (scale 0: every visible key weighs the same)."""
+    import torch
+    from paper_2608_10402_b200 import tide
+    HQ, HKV, D, S = 28, 4, 128, 16
+    rng = np.random.default_rng(31)
+    shapes = [(500, 1), (100, 90), (0, 300), (2100, 33)]
+    num_pages = sum((p + n + S - 1) // S for p, n in shapes) + 4
+    kv = tide.TideKV(HQ, HKV, D, S, num_pages, 4, 160, 4, 512)
+    orc = PagedKVOracle(num_pages, S, HKV, D, 4, 160)
+    cnt = [p + n for p, n in shapes]
+    indptr = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32)
+    T = int(indptr[-1])
+    k, v = inputs.normal_bf16(rng, (T, HKV, D)), inputs.normal_bf16(rng, (T, HKV, D))
+    for t in range(4):
+        kv.alloc(t)
+        orc.alloc(t)
+    kv.append(list(range(4)), indptr, H.to_dev(k, torch), H.to_dev(v, torch))
+    orc.append(list(range(4)), indptr, k, v)
+    rows = [(t, n, p + n) for t, (p, n) in enumerate(shapes)]
+    q = inputs.normal_bf16(rng, (sum(n for _, n in shapes), HQ, D))
+    out = torch.zeros((q.shape[0], HQ, D), dtype=torch.int16, device="cuda")
+    lse = torch.zeros((q.shape[0], HQ), dtype=torch.float32, device="cuda")
+    kv.attend(rows, H.to_dev(q, torch), scale, out, lse)
+    assert kv.status() == tide.OK
+    ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
+    H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, f"scale {scale}")
+    if scale == 0.0:
+        # closed form: LSE = ln(number of visible keys)
+        off = 0
+        for (p, n) in shapes:
+            want = np.log(np.arange(p + 1, p + n + 1, dtype=np.float64))
+            assert np.abs(lse[off:off + n].cpu().numpy() - want[:, None]).max() < 1e-4
+            off += n
+    kv.close()
