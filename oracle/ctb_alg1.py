@@ -16,9 +16,14 @@ Readings where the paper is silent (the same ones the product scheduler takes):
   * "fits in B_r": TokenUsage(r) + footprint(t) <= B_r;
   * "enforcing group affinity": a paused task may resume only on the rank it was preempted from (where its
     group's shared prefix lives); a task that never ran has no affinity;
-  * new tasks are considered in arrival order, the head of the queue only; it is admitted if its probed
-    footprint fits and the number of active tasks is below the environment-concurrency limit (the staleness and
-    task-diversity constraints need a trainer and task types and are not modelled);
+  * new tasks: "admit if it satisfies the constraints" (Section 4.2 lists policy staleness, task diversity and
+    environment concurrency).  Environment concurrency: the number of active tasks stays below `env_limit`.
+    Policy staleness ("throttles dispatch when Rollout is likely to generate more data than Trainer can consume
+    within the staleness bound"): no new task is admitted while the trajectories in flight - active, paused, and
+    finished but not yet consumed by the trainer (`unconsumed`, kept by the caller) - reach `inflight_cap`.
+    Task diversity ("penalizes assigning too many identical task types to the same batch"): among the first
+    `window` queued tasks whose probed footprint fits, the one whose type has the fewest active tasks on this
+    rank is admitted, ties in arrival order; window = 1 is plain arrival order;
   * ties in Priority go to the smaller task id;
   * a preempted task loses its KV state (Table 1: evicting long contexts costs a redundant prefill), so its
     footprint no longer counts against any rank.
@@ -36,6 +41,7 @@ class Task:
     group: int
     is_eval: bool
     probed: int                 # footprint estimated by the group's probing task (first turn)
+    kind: int = 0               # task type (environment), for the diversity constraint
     footprint: int = 0          # current token length (updated at the start of every interaction turn)
     state: str = "new"          # new | active | paused | done
     rank: int = -1              # rank it runs on (active) / was preempted from (paused)
@@ -60,7 +66,8 @@ def token_usage(tasks, r: int) -> int:
     return sum(t.footprint for t in tasks if t.state == "active" and t.rank == r)
 
 
-def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_limit: int, new_footprints=None):
+def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_limit: int, new_footprints=None,
+                  inflight_cap=None, unconsumed: int = 0, window: int = 1):
     """One iteration of the outer loop of Algorithm 1.
 
     tasks: list of Task (all of them); new_queue: list of task ids in arrival order (state "new");
@@ -93,12 +100,20 @@ def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_li
                 t_res.state = "active"
                 t_res.rank = r
                 events.append(("resume", t_res.id, r))
-            elif new_queue and n_active < env_limit and usage + by_id[new_queue[0]].probed <= B:
-                t_new = by_id[new_queue.pop(0)]
-                t_new.state = "active"
-                t_new.rank = r
-                t_new.footprint = t_new.probed
-                events.append(("admit", t_new.id, r))
             else:
-                break
+                # line 13: admit a new task if it satisfies the constraints
+                in_flight = sum(1 for t in tasks if t.state in ("active", "paused")) + unconsumed
+                fits = [tid for tid in new_queue[:window] if usage + by_id[tid].probed <= B]
+                if fits and n_active < env_limit and (inflight_cap is None or in_flight < inflight_cap):
+                    def same_kind_active(tid):
+                        return sum(1 for t in tasks if t.state == "active" and t.rank == r and t.kind == by_id[tid].kind)
+                    pick = min(fits, key=lambda tid: (same_kind_active(tid), new_queue.index(tid)))
+                    new_queue.remove(pick)
+                    t_new = by_id[pick]
+                    t_new.state = "active"
+                    t_new.rank = r
+                    t_new.footprint = t_new.probed
+                    events.append(("admit", t_new.id, r))
+                else:
+                    break
     return events

@@ -30,6 +30,7 @@ class CTBTask:
     group: int
     is_eval: bool
     probed: int
+    kind: int = 0
     footprint: int = 0
     state: str = "new"      # new | active | paused | done
     rank: int = -1
@@ -37,7 +38,7 @@ class CTBTask:
 
 class CTBScheduler:
     def __init__(self, budgets, weights=(8.0, 4.0, 2.0, 1.0), ctx_norm=8192.0, env_limit=1 << 30,
-                 on_admit=None, on_preempt=None, on_resume=None):
+                 on_admit=None, on_preempt=None, on_resume=None, inflight_cap=None, window=1):
         self.budgets = [int(b) for b in budgets]
         self.w_eval, self.w_group, self.w_active, self.w_ctx = (float(x) for x in weights)
         self.ctx_norm = float(ctx_norm)
@@ -51,11 +52,18 @@ class CTBScheduler:
         self.group_total = {}
         self.group_done = {}
         self.n_active = 0
+        # admission constraints of Section 4.2: policy staleness (no new task while active + paused + finished but
+        # unconsumed trajectories reach inflight_cap) and task diversity (among the first `window` queued tasks
+        # that fit, the type with the fewest active tasks on the rank goes first)
+        self.inflight_cap = inflight_cap
+        self.window = int(window)
+        self.unconsumed = 0
+        self.kind_active = [dict() for _ in self.budgets]   # per rank: task type -> active tasks
         self.on_admit, self.on_preempt, self.on_resume = on_admit, on_preempt, on_resume
 
     # ---- task life cycle ---------------------------------------------------------------------------------
-    def submit(self, task_id, group, probed, is_eval=False):
-        t = CTBTask(int(task_id), int(group), bool(is_eval), int(probed))
+    def submit(self, task_id, group, probed, is_eval=False, kind=0):
+        t = CTBTask(int(task_id), int(group), bool(is_eval), int(probed), int(kind))
         self.tasks[t.id] = t
         self.new_queue.append(t.id)
         self.group_total[t.group] = self.group_total.get(t.group, 0) + 1
@@ -68,10 +76,16 @@ class CTBScheduler:
             del self.active[t.rank][t.id]
             self.usage[t.rank] -= t.footprint
             self.n_active -= 1
+            self.kind_active[t.rank][t.kind] -= 1
         elif t.state == "paused":
             del self.paused[t.id]
         t.state = "done"
         self.group_done[t.group] += 1
+        self.unconsumed += 1
+
+    def consume(self, n):
+        """The trainer took n finished trajectories."""
+        self.unconsumed = max(0, self.unconsumed - int(n))
 
     def priority(self, t: CTBTask) -> float:
         return (self.w_eval * (1.0 if t.is_eval else 0.0)
@@ -94,6 +108,7 @@ class CTBScheduler:
                 del act[victim.id]
                 self.usage[r] -= victim.footprint
                 self.n_active -= 1
+                self.kind_active[r][victim.kind] -= 1
                 victim.state = "paused"
                 self.paused[victim.id] = victim
                 events.append(("evict", victim.id, r))
@@ -115,18 +130,37 @@ class CTBScheduler:
                     events.append(("resume", t.id, r))
                     if self.on_resume:
                         self.on_resume(t, r)
-                elif (self._new_head < len(self.new_queue) and self.n_active < self.env_limit
-                      and self.tasks[self.new_queue[self._new_head]].probed <= room):
-                    t = self.tasks[self.new_queue[self._new_head]]
-                    self._new_head += 1
+                else:
+                    pick = self._pick_new(r, room)
+                    if pick is None:
+                        break
+                    t = self.tasks[pick]
+                    if pick == self.new_queue[self._new_head]:
+                        self._new_head += 1
+                    else:
+                        self.new_queue.remove(pick)
                     t.footprint = t.probed
                     self._activate(t, r)
                     events.append(("admit", t.id, r))
                     if self.on_admit:
                         self.on_admit(t, r)
-                else:
-                    break
         return events
+
+    def _pick_new(self, r, room):
+        """The queued task to admit on rank r, or None: constraints of Section 4.2."""
+        if self._new_head >= len(self.new_queue) or self.n_active >= self.env_limit:
+            return None
+        if self.inflight_cap is not None and self.n_active + len(self.paused) + self.unconsumed >= self.inflight_cap:
+            return None
+        best = None
+        for pos in range(self._new_head, min(len(self.new_queue), self._new_head + self.window)):
+            tid = self.new_queue[pos]
+            t = self.tasks[tid]
+            if t.probed <= room:
+                key = (self.kind_active[r].get(t.kind, 0), pos)
+                if best is None or key < best[0]:
+                    best = (key, tid)
+        return None if best is None else best[1]
 
     def _activate(self, t, r):
         t.state = "active"
@@ -134,6 +168,7 @@ class CTBScheduler:
         self.active[r][t.id] = t
         self.usage[r] += t.footprint
         self.n_active += 1
+        self.kind_active[r][t.kind] = self.kind_active[r].get(t.kind, 0) + 1
 
     def pending_new(self):
         return len(self.new_queue) - self._new_head

@@ -7,11 +7,12 @@ from oracle import ctb_alg1 as oracle
 from paper_2608_10402_b200 import ctb
 
 
-def _trace(seed, n_ranks, passes=60):
+def _trace(seed, n_ranks, passes=60, inflight_cap=None, window=1, n_kinds=1):
     rng = np.random.default_rng(seed)
     budgets = [int(rng.integers(3000, 9000)) for _ in range(n_ranks)]
     env_limit = int(rng.integers(6, 30))
-    sched = ctb.CTBScheduler(budgets, ctx_norm=8192.0, env_limit=env_limit)
+    sched = ctb.CTBScheduler(budgets, ctx_norm=8192.0, env_limit=env_limit, inflight_cap=inflight_cap, window=window)
+    unconsumed = 0
     otasks, oqueue = [], []
     w = oracle.Weights()
     next_id = 0
@@ -19,8 +20,9 @@ def _trace(seed, n_ranks, passes=60):
         # arrivals
         for _ in range(int(rng.integers(0, 5))):
             group, is_eval, probed = int(rng.integers(0, 6)), bool(rng.random() < 0.15), int(rng.integers(200, 1500))
-            sched.submit(next_id, group, probed, is_eval)
-            otasks.append(oracle.Task(next_id, group, is_eval, probed))
+            kind = int(rng.integers(0, n_kinds))
+            sched.submit(next_id, group, probed, is_eval, kind=kind)
+            otasks.append(oracle.Task(next_id, group, is_eval, probed, kind=kind))
             oqueue.append(next_id)
             next_id += 1
         # some active tasks finish, the others grow (turn probing)
@@ -29,10 +31,16 @@ def _trace(seed, n_ranks, passes=60):
             if rng.random() < 0.1:
                 sched.finish(tid)
                 next(t for t in otasks if t.id == tid).state = "done"
+                unconsumed += 1
         grow = {tid: next(t for t in otasks if t.id == tid).footprint + int(rng.integers(0, 900))
                 for tid in act if next(t for t in otasks if t.id == tid).state == "active" and rng.random() < 0.7}
+        if inflight_cap is not None and rng.random() < 0.3:      # the trainer takes a batch
+            n = int(rng.integers(0, unconsumed + 1))
+            sched.consume(n)
+            unconsumed -= n
         got = sched.schedule(grow)
-        want = oracle.schedule_pass(otasks, oqueue, budgets, w, 8192.0, env_limit, grow)
+        want = oracle.schedule_pass(otasks, oqueue, budgets, w, 8192.0, env_limit, grow, inflight_cap=inflight_cap,
+                                    unconsumed=unconsumed, window=window)
         assert got == want, f"pass {p}: {got} != {want}"
         yield sched, otasks, budgets, env_limit, got
 
@@ -98,3 +106,36 @@ def test_simulated_rollout_ctb_keeps_more_kv_than_request_batching():
     # with ample memory nothing is ever dropped under either policy
     c = ctb.simulate(rollout, "request", 10**9, fixed_concurrency=96)
     assert c["hit_rate"] == 1.0
+
+
+def test_staleness_and_diversity_constraints_match_the_listing():
+    """Section 4.2's admission constraints: no new task while the trajectories in flight reach the cap; among the
+    first queued tasks that fit, the type least represented on the rank goes first."""
+    n_admit = 0
+    for seed in range(4):
+        cap = 10 + 3 * seed
+        for sched, otasks, budgets, env_limit, ev in _trace(100 + seed, n_ranks=1 + seed % 2, inflight_cap=cap, window=4, n_kinds=3):
+            n_admit += sum(1 for k, _, _ in ev if k == "admit")
+            in_flight = sum(1 for t in otasks if t.state in ("active", "paused")) + sched.unconsumed
+            # an admission happens only below the cap, so a pass can end at the cap but not beyond it through admissions
+            if any(k == "admit" for k, _, _ in ev):
+                assert in_flight <= cap
+            assert [t.id for t in otasks if t.state == "new"] == sched.new_queue[sched._new_head:]
+    assert n_admit > 30
+    # diversity on a hand-made case: rank 0 already runs two tasks of type 0; the queue holds types 0, 0, 1
+    s = ctb.CTBScheduler([100_000], window=3)
+    for i, kind in enumerate([0, 0]):
+        s.submit(i, group=i, probed=100, kind=kind)
+    s.schedule()
+    for i, kind in enumerate([0, 0, 1], start=2):
+        s.submit(i, group=i, probed=100, kind=kind)
+    assert [e[1] for e in s.schedule()] == [4, 2, 3]          # the type-1 task jumps the queue, then arrival order
+    # staleness on a hand-made case: cap 3, two active and one finished-but-unconsumed trajectory block admission
+    s = ctb.CTBScheduler([100_000], inflight_cap=3)
+    for i in range(5):
+        s.submit(i, group=i, probed=100)
+    assert [e[1] for e in s.schedule()] == [0, 1, 2]
+    s.finish(0)
+    assert s.schedule() == []                                  # 2 active + 1 unconsumed = cap
+    s.consume(1)
+    assert [e[1] for e in s.schedule()] == [3]
