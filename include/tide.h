@@ -218,6 +218,14 @@ int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k /*devic
  * bounded wait in a kernel ran out since the last call (the word is then cleared). */
 int tide_status(tide_kv_t* kv, void* stream);
 
+/* Rows of the most recently planned batch (tide_attend, tide_step_begin) that were planned as groups sharing their
+ * first pages: consecutive decode rows of distinct tasks whose page tables agree on at least 256 tokens of full
+ * pages (tasks made by tide_kv_fork).  The shared pages of a group are then read once for all its rows - the
+ * group's queries form one multi-query work item over them - and each row's own pages once, the two parts being
+ * combined by the same log-sum-exp merge that combines KV splits.  Results are those of tide_attend row by row
+ * (same tolerance); no grouping when the caller supplies its own page table. */
+int tide_last_sharing(tide_kv_t* kv, int64_t* groups, int64_t* rows);
+
 /* Counters of the most recent tide_attend: work items launched on the decode-style and the
  * tensor-tile paths, rows merged, and kernels launched by the most recent append + attend pair. */
 int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,

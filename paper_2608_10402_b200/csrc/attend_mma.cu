@@ -68,9 +68,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
   const int R = seg.n * g.G;                       // packed rows of this (row, kv head)
   const int tile_row0 = m_tile * TILE_M;
   const int r_last = min(R, tile_row0 + TILE_M) - 1;
-  const int kv_begin = split * seg.chunk;
-  const int kv_end = min(kv_begin + seg.chunk, seg.p + r_last / g.G + 1);
-  const bool direct = seg.n_splits == 1;
+  const int kv_begin = seg.origin + split * seg.chunk;
+  const int kv_end = min(kv_begin + seg.chunk, seg.p + (r_last / g.G) * seg.causal + 1);
+  const bool direct = seg.n_splits == 1 && seg.partial == 0;
   const float kLn2 = 0.6931471805599453f;
 
   // rows this thread owns inside its warp's 16-row MMA tile
@@ -137,16 +137,16 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
   }
 
   // ================= consumer warps =================
-  const int kv_limit_lo = v_lo ? min(kv_end, seg.p + qi_lo + 1) : kv_end;  // keys j < limit are visible
-  const int kv_limit_hi = v_hi ? min(kv_end, seg.p + qi_hi + 1) : kv_end;
+  const int kv_limit_lo = v_lo ? min(kv_end, seg.p + qi_lo * seg.causal + 1) : kv_end;  // keys j < limit are visible
+  const int kv_limit_hi = v_hi ? min(kv_end, seg.p + qi_hi * seg.causal + 1) : kv_end;
   // last key any row of this warp can see, and the smallest limit (masking needed beyond it)
   int w_end, w_min_limit;
   {
     const int wr_first = row_base, wr_last = min(R, row_base + 16) - 1;
     if (wr_last < wr_first) { w_end = kv_begin; w_min_limit = kv_end; }   // warp has no valid rows
     else {
-      w_end = min(kv_end, seg.p + wr_last / g.G + 1);
-      w_min_limit = min(kv_end, seg.p + wr_first / g.G + 1);
+      w_end = min(kv_end, seg.p + (wr_last / g.G) * seg.causal + 1);
+      w_min_limit = min(kv_end, seg.p + (wr_first / g.G) * seg.causal + 1);
     }
   }
 
@@ -423,18 +423,25 @@ __global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
   const int local = row - seg.merge_base;                 // token * Hq + head inside the segment
   const long long stride = (long long)seg.n * P.Hq;       // partial rows per split
   const long long p0 = seg.part_base + local;
+  // a row's contributions: its own splits, then (a member of a group that shares its first pages) the splits of the
+  // group's shared range, where this row is one token among the members' (such segments have one token: local = head)
+  const int n_src = seg.n_splits + seg.x_n_splits;
+  auto src_row = [&](int s) -> long long {
+    return s < seg.n_splits ? p0 + s * stride : (long long)seg.x_part_base + local + (long long)(s - seg.n_splits) * seg.x_stride;
+  };
   float mstar = -INFINITY;
-  for (int s = 0; s < seg.n_splits; ++s) mstar = fmaxf(mstar, P.part_lse[p0 + s * stride]);
+  for (int s = 0; s < n_src; ++s) mstar = fmaxf(mstar, P.part_lse[src_row(s)]);
   const float mu = (mstar == -INFINITY) ? 0.f : mstar;
   const int per = P.D / 32;                               // 2 or 4 floats per lane
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   float tot = 0.f;
-  for (int s = 0; s < seg.n_splits; ++s) {
-    const float e = P.part_lse[p0 + s * stride];
+  for (int s = 0; s < n_src; ++s) {
+    const long long pr = src_row(s);
+    const float e = P.part_lse[pr];
     if (e == -INFINITY) continue;
     const float w = exp2f(e - mu);
     tot += w;
-    const float* po = P.part_o + (p0 + s * stride) * P.D + lane * per;
+    const float* po = P.part_o + pr * P.D + lane * per;
     if (per == 4) {
       const float4 v = *reinterpret_cast<const float4*>(po);
       acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;

@@ -99,6 +99,7 @@ extern "C" int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const ti
       s.n_mtiles = 1;
       s.n_splits = n_splits;
       s.chunk = chunk;
+      s.causal = 1;
       if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
       segs[b] = s;
       qoff += r.q_len;

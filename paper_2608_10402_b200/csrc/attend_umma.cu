@@ -186,8 +186,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const int kvh = local / seg.n_splits;
   const int R = seg.n * g.G;
   const int item_row0 = m_tile * kUmmaTileRows * 2;
-  const int kv_begin = split * seg.chunk;
-  const bool direct = seg.n_splits == 1;
+  const int kv_begin = seg.origin + split * seg.chunk;
+  const bool direct = seg.n_splits == 1 && seg.partial == 0;
   // per 128-row tile: rows present, last key any of its rows sees, number of 64-key tiles to process
   int t_rows[2], t_end[2], t_tiles[2], t_min_limit[2];
 #pragma unroll
@@ -195,8 +195,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const int r0 = item_row0 + t * 128;
     t_rows[t] = max(0, min(128, R - r0));
     if (t_rows[t] > 0) {
-      t_end[t] = min(kv_begin + seg.chunk, seg.p + (r0 + t_rows[t] - 1) / g.G + 1);
-      t_min_limit[t] = min(t_end[t], seg.p + r0 / g.G + 1);
+      t_end[t] = min(kv_begin + seg.chunk, seg.p + ((r0 + t_rows[t] - 1) / g.G) * seg.causal + 1);
+      t_min_limit[t] = min(t_end[t], seg.p + (r0 / g.G) * seg.causal + 1);
       t_tiles[t] = t_end[t] > kv_begin ? (t_end[t] - kv_begin + kTileKeys - 1) / kTileKeys : 0;
     } else {
       t_end[t] = kv_begin; t_min_limit[t] = kv_begin; t_tiles[t] = 0;
@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const bool valid = r < R;
     const int qi = r / g.G, hd = kvh * g.G + (r - qi * g.G);
     const int my_tiles = t_tiles[t];
-    const int limit = valid ? min(t_end[t], seg.p + qi + 1) : t_end[t];   // keys j < limit are visible
+    const int limit = valid ? min(t_end[t], seg.p + qi * seg.causal + 1) : t_end[t];   // keys j < limit are visible
 
     // ---- this row of Q (or zeros) into TMEM as the A operand of S = Q.K^T: two bf16 per column ----
     {

@@ -24,6 +24,8 @@ constexpr int kSlotRecs = 2048;              // most append records per upload
 constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
 constexpr int kNumSms = 148;
 constexpr long long kPartRowsBase = 256 * 1024;
+constexpr long long kMinSavedBytesDefault = 64ll << 20;   // reads a batch must save before rows are planned as sharing groups
+constexpr int kStepSegStride = 2;   // each segment array of the step area holds up to 2 x max_batch_rows entries (rows + shared ranges)
 // header of the step area (int32 words): counts a fixed-shape launch reads on the device, as (count, segments) pairs
 constexpr int kHdrRecs = 0, kHdrDecItems = 2, kHdrTileItems = 4, kHdrUmmaItems = 6, kHdrMergeRows = 8;
 constexpr int kMaxHostChunks = 8;                 // most row groups of one host-buffer step
@@ -91,6 +93,9 @@ struct tide_kv {
   // last plan
   int64_t last_decode_items = 0, last_prefill_items = 0, last_merge_rows = 0, last_launches = 0;
   int64_t append_launches = 0;
+  int64_t last_groups = 0, last_grouped_rows = 0;   // rows planned as groups that share their first pages
+  bool no_grouping = false;
+  long long min_saved_bytes = kMinSavedBytesDefault;
   // optional per-phase timing (events on the caller's stream)
   bool profiling = false;
   cudaEvent_t ev_append[2] = {nullptr, nullptr};
@@ -151,10 +156,10 @@ Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
   L.off_old_row = off; off = align_up(off + (size_t)c->max_pages_per_task * 4 + 64, 256);   // row + one page pair
   // step area: 256-byte header of counts | write records | four segment arrays of max_batch_rows entries each
   L.step_seg_off = align_up(256 + (size_t)c->max_batch_rows * sizeof(AppendRec), 256);
-  L.step_bytes = align_up(L.step_seg_off + (size_t)(4 * c->max_batch_rows) * sizeof(Segment), 256);
+  L.step_bytes = align_up(L.step_seg_off + (size_t)(4 * kStepSegStride * c->max_batch_rows) * sizeof(Segment), 256);
   L.off_step = off; off += L.step_bytes;
   L.slot_bytes = align_up(256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8 + (size_t)kSlotRecs * 8 +
-                              (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);
+                              (size_t)(3 * c->max_batch_rows + 8) * sizeof(Segment), 256);   // rows + shared ranges (<= rows / 2) + merge list
   L.off_meta = off; off += L.slot_bytes * kSlots;
   L.part_rows = kPartRowsBase + (long long)g.Hq * c->max_batch_rows * 4;
   L.off_part_o = off; off = align_up(off + (size_t)L.part_rows * g.D * 4, 256);
@@ -309,6 +314,8 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->mark.assign((size_t)cfg->max_tasks, 0);
   kv->refcnt.assign((size_t)cfg->num_pages, 0);
   if (const char* e = getenv("TIDE_ITEMS_PER_SM")) kv->items_per_sm = std::max(1, atoi(e));  // tuning knob
+  if (const char* e = getenv("TIDE_NO_GROUPING")) kv->no_grouping = atoi(e) != 0;   // planner switch for comparisons
+  if (const char* e = getenv("TIDE_MIN_SAVED_BYTES")) kv->min_saved_bytes = atoll(e);  // tuning knob
   if (const char* e = getenv("TIDE_HOST_STEP_CHUNKS")) kv->host_step_chunks = std::max(0, atoi(e));  // tuning knob
   if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
@@ -824,51 +831,155 @@ static int check_rows(tide_kv* kv, int32_t n_rows, const tide_row_t* rows) {
   return TIDE_OK;
 }
 
+// Rows of one batch whose tasks hold the same first pages (forked tasks of a GRPO group, Section 2.1) are planned as
+// a group: consecutive decode rows of distinct tasks whose page lists agree on at least kMinSharedTokens tokens of
+// full pages that every member's context covers.
+struct ShareGroup {
+  int first = 0, m = 0, pages = 0;       // first member row, members, shared pages
+  int32_t part_base = 0, n_splits = 0;   // of the shared range's segment, known once it has been placed
+};
+constexpr int kMinSharedTokens = 256;
+
+constexpr int kMaxGroupRows = 64;        // packed rows of a shared range (one 64-row tile of the warp-MMA kernel, a quarter of a tcgen05 item)
+
+static void find_share_groups(const tide_kv* kv, int32_t n_rows, const tide_row_t* rows, std::vector<ShareGroup>& groups,
+                              std::vector<int>& group_of) {
+  const Geom& g = kv->g;
+  group_of.assign((size_t)n_rows, -1);
+  groups.clear();
+  const int max_m = std::max(1, kMaxGroupRows / g.G);
+  const int min_pages = std::max(1, kMinSharedTokens / g.S);
+  if (max_m < 2 || kv->no_grouping) return;
+  long long saved_total = 0;
+  for (int b = 0; b + 1 < n_rows; ++b) {
+    if (rows[b].q_len != 1) continue;
+    const auto& pg0 = kv->pages[rows[b].task];
+    int C = std::min<int>((int)pg0.size(), rows[b].ctx_len / g.S);
+    if (C < min_pages || kv->refcnt[(size_t)pg0[0]] < 2) continue;
+    int m = 1;
+    while (b + m < n_rows && m < max_m && rows[b + m].q_len == 1) {
+      const tide_row_t& r = rows[b + m];
+      bool repeat = false;
+      for (int k = 0; k < m; ++k) repeat = repeat || rows[b + k].task == r.task;
+      if (repeat) break;
+      const auto& pg = kv->pages[r.task];
+      const int lim = std::min<int>(std::min<int>(C, (int)pg.size()), r.ctx_len / g.S);
+      int lcp = 0;
+      while (lcp < lim && pg[(size_t)lcp] == pg0[(size_t)lcp]) ++lcp;
+      if (lcp < min_pages) break;
+      C = lcp;
+      ++m;
+    }
+    if (m >= 2) {
+      // Worth it only if the reads saved are a large part of what the members read: a group costs an extra work item
+      // for the shared range and a merge for every member (measured on 8 x 8 rows of 8192 keys: +8 % time at 12-25 %
+      // shared, break-even near 45 %, 1.4x faster at 75 %, 1.9x at 94 %).
+      long long ctx_sum = 0;
+      for (int k = 0; k < m; ++k) ctx_sum += rows[b + k].ctx_len;
+      const long long saved = (long long)(m - 1) * C * g.S;
+      if (saved * 10 >= ctx_sum * 4) {
+        ShareGroup sg;
+        sg.first = b; sg.m = m; sg.pages = C;
+        for (int k = 0; k < m; ++k) group_of[(size_t)(b + k)] = (int)groups.size();
+        groups.push_back(sg);
+        saved_total += saved;
+      }
+      b += m - 1;
+    }
+  }
+  // ... and only if the batch as a whole saves enough bytes to pay for one more kernel launch
+  if (saved_total * g.Hkv * g.D * 4 < kv->min_saved_bytes) {
+    groups.clear();
+    group_of.assign((size_t)n_rows, -1);
+  }
+}
+
 // The work plan of one batch: one segment per row, decode-style (<= 16 packed rows), warp-MMA tile-style or
 // tcgen05-style; long contexts are split along the keys so that the grid has about items_per_sm items per SM.
-// The plan depends on the rows only, so every layer of a step can use it.
-static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool umma_ok, PlanHost& P) {
+// A group of rows that share their first pages gets one more segment for the shared range (its tokens are the
+// members' queries, all seeing the same keys); the members' own segments start behind it and their merge takes both.
+// The plan depends on the rows and the page tables only, so every layer of a step can use it.
+static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool umma_ok, bool allow_groups, PlanHost& P) {
   const Geom& g = kv->g;
   enum { kDec = 0, kTile = 1, kUmma = 2 };
   struct RowPlan { int kind; int n_mtiles; long long items; };
+  auto kind_of = [&](int R) { return R <= kDecodeTileRows ? kDec : (umma_ok && R >= kv->umma_min_rows ? kUmma : kTile); };
+  auto mtiles_of = [&](int kind, int R) { return kind == kDec ? 1 : ceil_div(R, kind == kUmma ? 2 * kUmmaTileRows : kMmaTileRows); };
+  std::vector<ShareGroup> groups;
+  std::vector<int> group_of;
+  if (allow_groups) find_share_groups(kv, n_rows, rows, groups, group_of);
+  else group_of.assign((size_t)n_rows, -1);
   std::vector<RowPlan> plan((size_t)n_rows);
   long long w_dec = 0, w_tile = 0, items_tile_nosplit = 0;
   for (int b = 0; b < n_rows; ++b) {
     const tide_row_t& r = rows[b];
     const int R = r.q_len * g.G;
     RowPlan& p = plan[(size_t)b];
-    p.kind = R <= kDecodeTileRows ? kDec : (umma_ok && R >= kv->umma_min_rows ? kUmma : kTile);
-    p.n_mtiles = p.kind == kDec ? 1 : ceil_div(R, p.kind == kUmma ? 2 * kUmmaTileRows : kMmaTileRows);
+    p.kind = kind_of(R);
+    p.n_mtiles = mtiles_of(p.kind, R);
     p.items = (long long)g.Hkv * p.n_mtiles;
-    if (p.kind == kDec) w_dec += (long long)g.Hkv * r.ctx_len;
-    else { w_tile += p.items * r.ctx_len; items_tile_nosplit += p.items; }
+    const int own = group_of[(size_t)b] < 0 ? r.ctx_len : r.ctx_len - groups[(size_t)group_of[(size_t)b]].pages * g.S;
+    if (p.kind == kDec) w_dec += (long long)g.Hkv * own;
+    else { w_tile += p.items * own; items_tile_nosplit += p.items; }
   }
+  // A shared range is streaming work like a decode row (few rows against many keys), so it is cut as finely as
+  // decode rows are, whichever kernel its packed rows call for.
+  auto shared_kind = [&](int R) { return kind_of(R); };
+  for (const ShareGroup& sg : groups) w_dec += (long long)g.Hkv * sg.pages * g.S;
   const long long target = (long long)kNumSms * kv->items_per_sm;
   long long chunk_dec = std::max<long long>(256, align_up((size_t)(w_dec / target + 1), kStageKeys));
   long long chunk_tile = (items_tile_nosplit >= target / 2)
                              ? (1LL << 30)
                              : std::max<long long>(2048, align_up((size_t)(w_tile / target + 1), kStageKeys));
+  // a range of `len` keys cut for the given kind
+  auto cut = [&](bool streaming, int len, int& n_splits, int& chunk) {
+    const long long chunk_target = streaming ? chunk_dec : chunk_tile;
+    n_splits = (int)std::min<long long>(kMaxSplits, ((long long)len + chunk_target - 1) / chunk_target);
+    n_splits = std::max(1, n_splits);
+    chunk = (int)align_up((size_t)std::max(1, ceil_div(len, n_splits)), 2 * kStageKeys);
+    n_splits = std::max(1, ceil_div(len, chunk));
+  };
   for (int attempt = 0; attempt < 40; ++attempt) {
     P.seg_dec.clear(); P.seg_tile.clear(); P.seg_umma.clear();
     long long part_rows = 0, qoff = 0;
     for (int b = 0; b < n_rows; ++b) {
       const tide_row_t& r = rows[b];
       const RowPlan& p = plan[(size_t)b];
-      const long long chunk_target = p.kind == kDec ? chunk_dec : chunk_tile;
-      int n_splits = (int)std::min<long long>(kMaxSplits, ((long long)r.ctx_len + chunk_target - 1) / chunk_target);
-      n_splits = std::max(1, n_splits);
-      const int chunk = (int)align_up((size_t)ceil_div(r.ctx_len, n_splits), 2 * kStageKeys);
-      n_splits = ceil_div(r.ctx_len, chunk);
+      const int gi = group_of[(size_t)b];
+      if (gi >= 0 && groups[(size_t)gi].first == b) {
+        // the shared range of the group that starts at this row
+        const ShareGroup& sg = groups[(size_t)gi];
+        const int kind = shared_kind(sg.m * g.G);
+        Segment s{};
+        s.table_off = r.task * g.max_pages_per_task;
+        s.q_off = (int32_t)qoff;
+        s.n = sg.m;
+        s.p = sg.pages * g.S - 1;
+        s.n_mtiles = mtiles_of(kind, sg.m * g.G);
+        cut(true, sg.pages * g.S, s.n_splits, s.chunk);
+        s.causal = 0;
+        s.partial = 1;
+        s.x_part_base = gi;
+        s.x_n_splits = -2;                                   // marks the shared range until the links are resolved
+        part_rows += (long long)s.n_splits * sg.m * g.Hq;
+        (kind == kDec ? P.seg_dec : kind == kTile ? P.seg_tile : P.seg_umma).push_back(s);
+      }
       Segment s{};
       s.table_off = r.task * g.max_pages_per_task;
       s.q_off = (int32_t)qoff;
       s.n = r.q_len;
       s.p = r.ctx_len - r.q_len;
       s.n_mtiles = p.n_mtiles;
-      s.n_splits = n_splits;
-      s.chunk = chunk;
-      s.part_base = 0;
-      if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
+      s.causal = 1;
+      if (gi >= 0) {
+        s.origin = groups[(size_t)gi].pages * g.S;
+        s.partial = 1;
+        s.x_part_base = gi;
+        s.x_n_splits = -1;                                   // marks a member until the links are resolved
+        s.x_stride = b - groups[(size_t)gi].first;           // member index, for now
+      }
+      cut(p.kind == kDec, r.ctx_len - s.origin, s.n_splits, s.chunk);
+      if (s.n_splits > 1 || s.partial) part_rows += (long long)s.n_splits * r.q_len * g.Hq;
       (p.kind == kDec ? P.seg_dec : p.kind == kTile ? P.seg_tile : P.seg_umma).push_back(s);
       qoff += r.q_len;
     }
@@ -879,7 +990,7 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
   }
   // heaviest items first, so the tail of the grid is made of short items
   auto heavier = [](const Segment& a, const Segment& b) {
-    return std::min(a.chunk, a.p + a.n) > std::min(b.chunk, b.p + b.n);
+    return std::min(a.chunk, a.p + a.n - a.origin) > std::min(b.chunk, b.p + b.n - b.origin);
   };
   std::stable_sort(P.seg_dec.begin(), P.seg_dec.end(), heavier);
   std::stable_sort(P.seg_tile.begin(), P.seg_tile.end(), heavier);
@@ -887,22 +998,46 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
   P.seg_merge.clear();
   P.merge_rows = 0;
   long long part_cursor = 0;
+  std::vector<Segment*> merged;                              // segments with rows to merge, in merge_base order
   for (auto* v : {&P.seg_dec, &P.seg_tile, &P.seg_umma}) {
     long long base = 0;
     for (Segment& s : *v) {
       s.item_base = (int32_t)base;
       base += (long long)g.Hkv * s.n_mtiles * s.n_splits;
       if (base > 0x7fffffffLL) return TIDE_ERR_WORKSPACE;
-      if (s.n_splits > 1) {
+      if (s.n_splits > 1 || s.partial) {
         s.part_base = (int32_t)part_cursor;
         part_cursor += (long long)s.n_splits * s.n * g.Hq;
-        s.merge_base = (int32_t)P.merge_rows;
-        P.merge_rows += (long long)s.n * g.Hq;
-        P.seg_merge.push_back(s);
+        if (s.x_n_splits == -2) {                            // a shared range: it has no output rows of its own
+          groups[(size_t)s.x_part_base].part_base = s.part_base;
+          groups[(size_t)s.x_part_base].n_splits = s.n_splits;
+        } else {
+          s.merge_base = (int32_t)P.merge_rows;
+          P.merge_rows += (long long)s.n * g.Hq;
+          merged.push_back(&s);
+        }
       }
     }
     (v == &P.seg_dec ? P.items_dec : v == &P.seg_tile ? P.items_tile : P.items_umma) = base;
   }
+  // resolve the links between the members and their group's shared range
+  for (auto* v : {&P.seg_dec, &P.seg_tile, &P.seg_umma})
+    for (Segment& s : *v) {
+      if (s.x_n_splits == -1) {
+        const ShareGroup& sg = groups[(size_t)s.x_part_base];
+        const int member = s.x_stride;
+        s.x_part_base = sg.part_base + member * g.Hq;
+        s.x_n_splits = sg.n_splits;
+        s.x_stride = sg.m * g.Hq;
+      } else if (s.x_n_splits == -2) {
+        s.x_part_base = 0;
+        s.x_n_splits = 0;
+      }
+    }
+  for (const Segment* s : merged) P.seg_merge.push_back(*s);
+  kv->last_groups = (int64_t)groups.size();
+  kv->last_grouped_rows = 0;
+  for (const ShareGroup& sg : groups) kv->last_grouped_rows += sg.m;
   return TIDE_OK;
 }
 
@@ -990,7 +1125,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   int rc = check_rows(kv, n_rows, rows);
   if (rc != TIDE_OK) return rc;
   PlanHost P;
-  if ((rc = build_plan(kv, n_rows, rows, kv->g.D == 128 && scale > 0.f, P)) != TIDE_OK) return rc;
+  if ((rc = build_plan(kv, n_rows, rows, kv->g.D == 128 && scale > 0.f, page_table == nullptr, P)) != TIDE_OK) return rc;
   if (P.n_all() * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
 
   cudaStream_t st = (cudaStream_t)stream;
@@ -1045,7 +1180,7 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
   // The plan needs the lengths after the step only through ctx_len, which the rows already carry, so it is built
   // (and can still be refused) before anything changes.
   PlanHost P;
-  if ((rc = build_plan(kv, n_rows, rows, g.D == 128, P)) != TIDE_OK) return rc;
+  if ((rc = build_plan(kv, n_rows, rows, g.D == 128, true, P)) != TIDE_OK) return rc;
   if (kv->fixed_grids && (P.items_dec > kv->cap_dec || P.items_tile > kv->cap_tile || P.items_umma > kv->cap_umma ||
                           P.merge_rows > kv->cap_merge_rows || indptr[(size_t)n_rows] > kv->cap_tokens))
     return TIDE_ERR_WORKSPACE;   // the step does not fit the launch shapes that were fixed
@@ -1068,7 +1203,7 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
     recs[b].count = rows[b].q_len;
   }
   uint8_t* d_step = kv->ws + kv->lay.off_step;
-  const size_t stride = (size_t)kv->cfg.max_batch_rows;
+  const size_t stride = (size_t)kStepSegStride * (size_t)kv->cfg.max_batch_rows;
   kv->step_plan = pack_plan(P, (Segment*)(kv->h_step + kv->lay.step_seg_off), (const Segment*)(d_step + kv->lay.step_seg_off), stride);
   // header and records in one copy, then each segment array that is not empty (their places are fixed)
   if (cudaMemcpyAsync(d_step, kv->h_step, 256 + (size_t)n_rows * sizeof(AppendRec), cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -1285,6 +1420,13 @@ int tide_internal_view(tide_kv_t* kv, Geom* g, const uint8_t** pool, const int32
   *len = kv->len.data();
   *live = kv->live.data();
   *max_tasks = kv->cfg.max_tasks;
+  return TIDE_OK;
+}
+
+int tide_last_sharing(tide_kv_t* kv, int64_t* groups, int64_t* rows) {
+  if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
+  if (groups) *groups = kv->last_groups;
+  if (rows) *rows = kv->last_grouped_rows;
   return TIDE_OK;
 }
 

@@ -41,11 +41,19 @@ struct __align__(16) Segment {
   int32_t n_mtiles;
   int32_t n_splits;
   int32_t chunk;       // keys per split, a multiple of kStageKeys
-  int32_t part_base;   // first partial row ((split * n + token) * Hq + head) when n_splits > 1
+  int32_t part_base;   // first partial row ((split * n + token) * Hq + head) when the item writes partials
   int32_t merge_base;  // first row of this segment in the merge launch
-  int32_t pad0, pad1;
+  // Rows of one batch whose tasks share their first pages (forked tasks) read those pages once: the shared range
+  // is one segment whose `n` tokens are the member rows' queries and all see the same keys (causal = 0), each
+  // member's own range starts behind it (origin), both write partials, and the member's merge takes both.
+  int32_t causal;      // query i sees keys [0, p + i * causal + 1): 1 for a task's own tokens, 0 for a shared range
+  int32_t origin;      // first key of the range this segment covers (split s starts at origin + s * chunk)
+  int32_t partial;     // 1: write partials even when n_splits == 1 (another segment contributes to the same rows)
+  int32_t x_part_base; // the other contribution to this segment's rows: first partial row of token 0's head 0 ...
+  int32_t x_n_splits;  // ... its number of splits (0 = none) ...
+  int32_t x_stride;    // ... and the distance in rows between its consecutive splits
 };
-static_assert(sizeof(Segment) == 48, "Segment layout");
+static_assert(sizeof(Segment) == 64, "Segment layout");
 
 struct AttendParams {
   const uint8_t* pool;

@@ -47,7 +47,7 @@ EXPORTS = [
     "tide_kv_alloc", "tide_kv_append", "tide_attend", "tide_step_host", "tide_kv_release", "tide_kv_truncate",
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
     "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune", "tide_kv_fork", "tide_kv_page_refs",
-    "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer", "tide_step_fix_grids",
+    "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer", "tide_step_fix_grids", "tide_last_sharing",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -265,6 +265,11 @@ class TideKV:
         v = [ctypes.c_float(0) for _ in range(4)]
         _check(lib.tide_phase_ms(self.handle, *[ctypes.byref(x) for x in v]), "tide_phase_ms")
         return {"append": v[0].value, "decode": v[1].value, "tile": v[2].value, "merge": v[3].value}
+
+    def last_sharing(self):
+        a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib.tide_last_sharing(self.handle, ctypes.byref(a), ctypes.byref(b)), "tide_last_sharing")
+        return {"groups": a.value, "rows": b.value}
 
     def last_plan(self):
         a, b, c, d = (ctypes.c_int64(0) for _ in range(4))

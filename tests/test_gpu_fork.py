@@ -127,3 +127,79 @@ def test_random_ops_with_forks_match_the_oracle_bit_for_bit():
     _same(kv, orc, sorted(orc.live))
     assert codes["fork"] > 5 and codes["errors"] > 3, codes
     kv.close()
+
+
+@pytest.mark.parametrize("geom", [(28, 4, 128, 16), (8, 2, 64, 16), (16, 1, 128, 32), (4, 4, 64, 32)])
+def test_decode_rows_of_forked_groups_read_their_shared_pages_once(geom, monkeypatch):
+    """Groups of trajectories forked from one prompt, then decoding: the planner must treat each group's shared
+    pages as one multi-query range (tide_last_sharing), and every row's result must still be plain attention over
+    its whole context.  Group sizes around what one work item holds, members with and without tokens of their
+    own, one unshared task in between, a context that ends inside the shared pages."""
+    import torch
+    from paper_2608_10402_b200 import tide
+    HQ, HKV, D, S = geom
+    monkeypatch.setenv("TIDE_MIN_SAVED_BYTES", "0")      # small test batches: no minimum saving per batch
+    rng = np.random.default_rng(HQ + D + S)
+    scale = 1.0 / math.sqrt(D)
+    NT = 40
+    kv = tide.TideKV(HQ, HKV, D, S, 2000, NT, 200, NT, 64)
+    orc = PagedKVOracle(2000, S, HKV, D, NT, 200)
+
+    def app(ts, cnt):
+        ip = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int32)
+        T = int(ip[-1])
+        k, v = inputs.normal_bf16(rng, (T, HKV, D)), inputs.normal_bf16(rng, (T, HKV, D))
+        kv.append(ts, ip, H.to_dev(k, torch), H.to_dev(v, torch))
+        orc.append(ts, ip, k, v)
+
+    task = 0
+    rows_tasks = []
+    for prompt, members, own in [(1500, 8, True), (700, 3, True), (4 * S * 16, 12, False), (300, 2, True)]:
+        lead = task
+        for o in (kv, orc):
+            o.alloc(lead)
+        app([lead], [prompt])
+        ids = [lead]
+        for _ in range(members - 1):
+            task += 1
+            kv.fork(lead, task)
+            orc.fork(lead, task)
+            ids.append(task)
+        task += 1
+        if own:
+            app(ids, [int(rng.integers(1, 90)) for _ in ids])      # every trajectory continues on its own
+        rows_tasks += ids
+        if members == 3:                                            # an unshared task between two groups
+            for o in (kv, orc):
+                o.alloc(task)
+            app([task], [900])
+            rows_tasks.append(task)
+            task += 1
+    # one decode step: every task appends a token
+    app(rows_tasks, [1] * len(rows_tasks))
+    rows = [(t, 1, orc.task_len(t)) for t in rows_tasks]
+    q = inputs.normal_bf16(rng, (len(rows), HQ, D))
+    out = torch.zeros((len(rows), HQ, D), dtype=torch.int16, device="cuda")
+    lse = torch.zeros((len(rows), HQ), dtype=torch.float32, device="cuda")
+    kv.attend(rows, H.to_dev(q, torch), scale, out, lse)
+    assert kv.status() == tide.OK
+    ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
+    H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, f"grouped decode {geom}")
+    sharing = kv.last_sharing()
+    assert sharing["groups"] >= 3 and sharing["rows"] >= 8 + 3 + 4, sharing
+    # a window that ends inside the shared pages, and windows shorter than the shared range, still come out right
+    rows2 = [(t, 1, max(1, min(orc.task_len(t), int(rng.integers(1, 1600))))) for t in rows_tasks]
+    kv.attend(rows2, H.to_dev(q, torch), scale, out, lse)
+    assert kv.status() == tide.OK
+    ref_o, ref_l = cbuild.attend_paged(orc, rows2, q, scale)
+    H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, f"grouped decode, windows {geom}")
+    # with the caller's own page table there is no grouping, and the result is the same attention
+    table = torch.zeros((NT, 200), dtype=torch.int32, device="cuda")
+    for t in rows_tasks:
+        pt = orc.page_table(t)
+        table[t, :len(pt)] = torch.from_numpy(pt).cuda()
+    kv.attend(rows, H.to_dev(q, torch), scale, out, lse, page_table=table)
+    assert kv.last_sharing()["groups"] == 0
+    ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
+    H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, f"own table {geom}")
+    kv.close()
