@@ -239,3 +239,27 @@ def test_step_host_matches_append_then_attend(env, groups, monkeypatch):
     ref_o, ref_l = H.oracle_attend(c, w, q_bits)
     H.check_outputs(hout.numpy().view(np.uint16), hlse.numpy(), ref_o, ref_l, "step_host")
     kv.close()
+
+
+def test_outputs_are_bitwise_independent_of_where_the_pages_lie(env):
+    """The plan depends on logical lengths only and no kernel's arithmetic order depends on page numbers, so the
+    same batch over two different page permutations (and run twice) must give the same bits, not just the same
+    values within tolerance."""
+    tide, torch = env
+    w = inputs.make_workload(3, n_tasks=12, len_div=8)
+    kv_bits = [w.task_kv(b) for b in range(w.B)]
+    q_bits = np.concatenate([w.task_q(b) for b in range(w.B)])
+    _, indptr, nk, nv = H.oracle_fill(w, kv_bits)
+    total_q = q_bits.shape[0]
+    results = []
+    for seed in (1, 2, 2):
+        w.free_order = np.random.default_rng(seed).permutation(w.num_pages).astype(np.int32)
+        kv = H.gpu_fill(w, kv_bits, nk, nv, indptr, tide, torch)
+        out = torch.zeros((total_q, w.Hq, w.D), dtype=torch.int16, device="cuda")
+        lse = torch.zeros((total_q, w.Hq), dtype=torch.float32, device="cuda")
+        kv.attend(w.rows(), H.to_dev(q_bits, torch), w.scale, out, lse)
+        assert kv.status() == tide.OK
+        results.append((out.cpu().numpy().copy(), lse.cpu().numpy().copy()))
+        kv.close()
+    for o, l in results[1:]:
+        assert np.array_equal(o, results[0][0]) and np.array_equal(l.view(np.uint32), results[0][1].view(np.uint32))
