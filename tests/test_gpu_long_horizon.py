@@ -173,8 +173,8 @@ def test_long_horizon_release_and_reuse():
             next_task += 1
         assert reused > 0, "released pages were not handed out again"
         assert kv.usage() == (orc.used_tokens(), orc.free_pages())
-    out_dir = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(out_dir):
+    out_dir = os.environ.get("TIDE_REPORT_DIR", "")
+    if out_dir and os.path.isdir(out_dir):
         with open(os.path.join(out_dir, f"long_horizon_{int(report['pool_gb'])}gb.json"), "w") as f:
             json.dump(report, f, indent=1)
     print(json.dumps({k: v for k, v in report.items() if k != "steps"}), [round(s["ms"], 3) for s in report["steps"]])
