@@ -9,8 +9,8 @@
 // This is a dense contraction (n*G x ctx x D), so it is bound by the tensor pipe: 4*D flops per visible
 // (packed row, key) pair against Hkv*D*4 bytes per key shared by all packed rows.
 //
-// CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warp 8 streams K
-// and V tiles of 64 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
+// CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warps 8, 10 and 11
+// stream K and V tiles of 64 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
 // 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.  TMEM (512 columns):
 //   Q_A Q_B   2 x 64   the queries as packed bf16, staged once per item
 //   S_A S_B   2 x 64   fp32 logits of one 64-key tile; P (packed bf16) overwrites the first 32 columns
@@ -33,8 +33,9 @@ namespace umma {
 
 constexpr int D = 128;
 constexpr int kTileKeys = 64;
-constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA issuer, 2 idle warps}
+constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {three producer warps and the MMA issuer}
 constexpr int kNumBuf = 6;                          // ring of (K tile, V tile) slots
+constexpr int kProducerWarps = 3;                   // warps 8, 10, 11
 constexpr int kTileBytes = kTileKeys * D * 2;       // one K or V tile: 16 KB
 constexpr int kSlotBytes = 2 * kTileBytes;          // K tile then V tile
 constexpr int kSlabBytes = kTileKeys * 128;         // 64 rows x 128 bytes
@@ -213,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
+    for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), kProducerWarps); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
     mbar_init(smem_u32(&bars.q_full), 256);
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
@@ -237,8 +238,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   // more than that: 256 x 224 + 128 x 56 = 384 x 168.  (An over-subscribed .inc waits for ever.)
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    if (warp == 8) {
-      // ================= producer: K0 V0 K1 V1 ... into the ring =================
+    if (warp != 9) {
+      // ================= producers: K0 V0 K1 V1 ... into the ring =================
+      // Three warps (8, 10, 11) share the copies of every tile: a bulk copy costs its warp about 55 cycles of
+      // issue whatever its size, so the 16 copies of a tile from one warp (~1400 cycles per 32 KB measured) were
+      // most of a tile pair's time; each warp announces its own bytes on the slot's barrier.
+      const int pw = warp == 8 ? 0 : warp - 9;                 // 0, 1, 2
       if (n_tiles > 0) {
         const int pages_per_tile = kTileKeys / g.S;
         const int slab_block = g.S * 128;                    // bytes of one slab of a page block
@@ -261,18 +266,20 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           const int key0 = kv_begin + j * kTileKeys;
           const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
           const uint32_t bar = smem_u32(&bars.kv_full[buf]);
-          if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * 4 * slab_block));
-          // lanes [0, copies) fetch the K pieces, lanes [copies, 2*copies) the V pieces of this tile
+          // lanes [0, copies) fetch the K pieces, lanes [copies, 2*copies) the V pieces of this tile; every third one here
           const int is_v = lane >= copies ? 1 : 0;
           const int c = lane - is_v * copies;
           const int pg = c >> 1, slab = c & 1;
           const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + pg) & 31);
-          if (lane < 2 * copies && pg < npages) {
+          const bool mine = lane < 2 * copies && pg < npages && lane % kProducerWarps == pw;
+          const uint32_t n_mine = (uint32_t)__popc(__ballot_sync(0xffffffffu, mine));
+          if (lane == 0) mbar_expect_tx(bar, n_mine * (uint32_t)slab_block);
+          if (mine) {
             const uint8_t* src = P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes + is_v * g.kblock_bytes + slab * slab_block;
             bulk_g2s(smem_base + buf * kSlotBytes + is_v * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
           }
         }
-        if (*abort_flag && lane == 0) {
+        if (*abort_flag && lane == 0 && pw == 0) {
           // a wait gave up somewhere: do not leave while copies into this CTA's shared memory are in flight
           for (int idx = max(0, n_tiles - kNumBuf); idx < n_tiles; ++idx) {
             const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
