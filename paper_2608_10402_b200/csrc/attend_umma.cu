@@ -118,6 +118,25 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// packed pairs of floats: one instruction for two elements (fma.rn.f32x2 / add.rn.f32x2)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -454,16 +473,24 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       const float mu = (m == -INFINITY) ? 0.f : m;
       float sp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
+      // packed arithmetic: the softmax warps are short of issue slots, and this halves the scale-subtract and the
+      // row-sum instructions (same roundings and the same summation order as the scalar form)
+      {
+        const uint64_t sl2_2 = pack2(sl2, sl2), nmu_2 = pack2(-mu, -mu);
+        uint64_t sp2[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
-      for (int c = 0; c < 64; c += 8) {
+        for (int c = 0; c < 64; c += 8) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float e = fast_exp2(fmaf(s[c + i], sl2, -mu));
-          s[c + i] = e;
-          sp[i] += e;
+          for (int i = 0; i < 4; ++i) {
+            float x0, x1;
+            unpack2(fma2(pack2(s[c + 2 * i], s[c + 2 * i + 1]), sl2_2, nmu_2), x0, x1);
+            const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
+            sp2[i] = add2(sp2[i], pack2(e0, e1));
+            pk[(c >> 1) + i] = pack_bf16(e0, e1);
+          }
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) pk[(c >> 1) + i] = pack_bf16(s[c + 2 * i], s[c + 2 * i + 1]);
+        for (int i = 0; i < 4; ++i) unpack2(sp2[i], sp[2 * i], sp[2 * i + 1]);
       }
       TT_PH(2);
       tmem_st32u(s_addr, pk);                                  // P_t over the first 32 columns of S_t
