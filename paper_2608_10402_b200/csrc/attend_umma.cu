@@ -24,6 +24,7 @@
 // more than 2^8 (the final normalisation uses the same stale maximum, so the result is exact).
 // Every wait is bounded; a wait that runs out sets TIDE_ERR_DEVICE_TIMEOUT and the CTA drains and exits.
 #include <climits>
+#include <type_traits>
 
 #include "tide_internal.h"
 
@@ -422,7 +423,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 
     TT_DECL;
     TT_PH_DECL;
-    for (int j = 0; j < my_tiles; ++j) {
+    // One key tile of this row tile.  The tiles that need the causal (or end-of-range) mask are the last ones of the
+    // item; they get a copy of the body of their own, so the 128 compare-and-select instructions of the mask are
+    // not part of the code that the other ~99 % of the tiles run (its mere presence in the loop cost 2 %).
+    auto tile = [&](const int j, auto masked_tag) {
+      constexpr bool kMasked = decltype(masked_tag)::value;
       TT_BEGIN;
       mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
       TT_END(tt_wait);
@@ -433,9 +438,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       tmem_ld32(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_wait_ld();
       TT_PH(0);
-      const int tile_key0 = kv_begin + j * kTileKeys;
-      if (tile_key0 + kTileKeys > t_min_limit[t]) {            // uniform over the warpgroup
-        const int vis = limit - tile_key0;
+      if constexpr (kMasked) {
+        const int vis = limit - (kv_begin + j * kTileKeys);
 #pragma unroll
         for (int c = 0; c < 64; ++c) if (c >= vis) s[c] = -INFINITY;
       }
@@ -499,7 +503,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       tc_fence_before();
       mbar_arrive(smem_u32(&bars.p_full[t]));
       TT_PH(3);
-    }
+    };
+    // tiles j < n_plain end at or before the first row's limit: every key of theirs is visible to every row
+    const int n_plain = min(my_tiles, max(0, (t_min_limit[t] - kv_begin) / kTileKeys));
+    for (int j = 0; j < n_plain; ++j) tile(j, std::false_type{});
+    for (int j = n_plain; j < my_tiles; ++j) tile(j, std::true_type{});
 
     // ---- epilogue: O / l and LSE ----
     const float kLn2 = 0.6931471805599453f;
