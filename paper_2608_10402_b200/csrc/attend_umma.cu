@@ -457,19 +457,21 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       float mx = max3(max3(mxp[0], mxp[1], mxp[2]), max3(mxp[3], mxp[4], mxp[5]), fmaxf(mxp[6], mxp[7]));
       mx *= sl2;                                               // scale > 0 on this path
       float m_new = m;
-      if (mx > m + kRescaleThreshold || m == -INFINITY) m_new = fmaxf(m, mx);
+      if (mx > m + kRescaleThreshold) m_new = mx;             // also the first visible key: -inf + 8 = -inf < any finite mx
       float alpha = 1.f;
-      if (__any_sync(0xffffffffu, m_new != m)) alpha = fast_exp2(m - m_new);   // rare; m = -inf -> 0, equal -> 1
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-        // O_t holds tiles < j: S_t(j) was committed after PV_t(j-1)
+      if (__any_sync(0xffffffffu, m_new != m)) {               // rare: one vote per tile decides both steps
+        alpha = fast_exp2(m - m_new);                          // m = -inf -> 0, equal -> 1
+        if (j > 0) {
+          // O_t holds tiles < j: S_t(j) was committed after PV_t(j-1)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          float o[32];
-          tmem_ld32(o_addr + c * 32, o);
-          tmem_wait_ld();
+          for (int c = 0; c < 4; ++c) {
+            float o[32];
+            tmem_ld32(o_addr + c * 32, o);
+            tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] *= alpha;
-          tmem_st32(o_addr + c * 32, o);
+            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+            tmem_st32(o_addr + c * 32, o);
+          }
         }
       }
       m = m_new;
