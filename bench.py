@@ -31,7 +31,7 @@ METRIC = "mixed resume batch: KV-read GB/s vs HBM peak; append-prefill TFLOP/s v
 # scaled by the units one launch processes): decode kernel dram bytes / algorithmic KV bytes; tcgen05 kernel
 # dram bytes per flop of resume-row attention.
 NCU_DECODE_TRAFFIC_RATIO = 1.011
-NCU_UMMA_DRAM_BYTES_PER_FLOP = 350.7e6 / 863.8e9
+NCU_UMMA_DRAM_BYTES_PER_FLOP = 348.6e6 / 863.8e9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
