@@ -1,34 +1,36 @@
 """Oracle for the paper's Algorithm 1, "Semantic-Aware CTB Scheduling" (test infrastructure only).
 
-One scheduling pass, written in the order and notation of the listing: update the token footprints of the
-active tasks; then for each rank r, while TokenUsage(r) exceeds the budget B_r preempt the active task of r with
-the lowest Priority; while TokenUsage(r) is below B_r resume the paused task with the highest Priority that fits
-(enforcing group affinity), otherwise admit a new task by its probed footprint if it satisfies the constraints,
-otherwise stop.  Priority is the unnumbered equation of Section 4.2,
+One scheduling pass in the algorithm's own order of steps and with its names.  First the token footprints of
+the active tasks are refreshed from turn probing.  Then every rank r is visited in turn: as long as
+TokenUsage(r) is above the budget B_r, the active task of r with the smallest Priority is preempted; after that,
+as long as TokenUsage(r) is below B_r, the rank is filled - a paused task that fits goes first (the one with the
+largest Priority, subject to group affinity), a new task is admitted by its probed footprint only when no paused
+task can be resumed and the admission constraints hold, and the fill loop ends when neither is possible.
+Priority is the weighted sum of Section 4.2,
 
     P(t) = w1 * I_eval + w2 * G_completion + w3 * I_active + w4 * L_context .
 
-Readings where the paper is silent (the same ones the product scheduler takes):
-  * weights: the paper gives none; the caller passes them (the tests use 8, 4, 2, 1, which reproduces the strict
+Readings where the paper is silent:
+  * weights: the paper gives none; the caller passes them (the tests use 8, 4, 2, 1, which gives the strict
     tiers of Table 1 because every factor lies in [0, 1]);
-  * L_context is the task's current token length divided by `ctx_norm` (so that it lies in [0, 1]);
-  * G_completion = finished / total of the task's GRPO group;
-  * "fits in B_r": TokenUsage(r) + footprint(t) <= B_r;
-  * "enforcing group affinity": a paused task may resume only on the rank it was preempted from (where its
-    group's shared prefix lives); a task that never ran has no affinity;
-  * new tasks: "admit if it satisfies the constraints" (Section 4.2 lists policy staleness, task diversity and
-    environment concurrency).  Environment concurrency: the number of active tasks stays below `env_limit`.
-    Policy staleness ("throttles dispatch when Rollout is likely to generate more data than Trainer can consume
-    within the staleness bound"): no new task is admitted while the trajectories in flight - active, paused, and
-    finished but not yet consumed by the trainer (`unconsumed`, kept by the caller) - reach `inflight_cap`.
-    Task diversity ("penalizes assigning too many identical task types to the same batch"): among the first
-    `window` queued tasks whose probed footprint fits, the one whose type has the fewest active tasks on this
-    rank is admitted, ties in arrival order; window = 1 is plain arrival order;
+  * L_context is the task's current token length divided by `ctx_norm`, capped at 1;
+  * G_completion = finished / total members of the task's GRPO group;
+  * a task "fits" when TokenUsage(r) + footprint(t) <= B_r;
+  * group affinity: a paused task may resume only on the rank it was preempted from (where its group's shared
+    prefix lives); a task that never ran has no affinity;
+  * the admission constraints of Section 4.1.  Environment concurrency: the number of active tasks stays below
+    `env_limit`, for resumes and admissions alike.  Policy staleness: no new task is admitted while the
+    trajectories in flight - active, paused, and finished but not yet taken by the trainer (`unconsumed`, kept by
+    the caller) - have reached `inflight_cap`.  Task diversity: among the first `window` queued tasks whose
+    probed footprint fits, the one whose type has the fewest active tasks on this rank is admitted, ties in
+    arrival order; window = 1 is plain arrival order;
   * ties in Priority go to the smaller task id;
-  * a preempted task loses its KV state (Table 1: evicting long contexts costs a redundant prefill), so its
-    footprint no longer counts against any rank.
+  * a preempted task loses its KV state (Table 1 counts the prefill it will have to repeat as the cost of
+    evicting a long context), so its footprint no longer counts against any rank.
 
-Everything is plain Python over lists: no heaps, no incremental sums.
+Everything is plain Python over lists, recomputed from scratch at every use: no heaps, no running sums.
+Pinned in tests/test_ctb_scheduler.py by hand-derived decision lists (tier order, affinity over two ranks,
+resume before admit, the three admission constraints) and by the invariants the loop guarantees.
 """
 from __future__ import annotations
 
@@ -68,7 +70,7 @@ def token_usage(tasks, r: int) -> int:
 
 def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_limit: int, new_footprints=None,
                   inflight_cap=None, unconsumed: int = 0, window: int = 1):
-    """One iteration of the outer loop of Algorithm 1.
+    """One pass of Algorithm 1 over all ranks.
 
     tasks: list of Task (all of them); new_queue: list of task ids in arrival order (state "new");
     budgets: B_r per rank; new_footprints: {task id: tokens} from turn probing.
@@ -76,13 +78,12 @@ def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_li
     ("evict", task, rank) | ("resume", task, rank) | ("admit", task, rank)."""
     by_id = {t.id: t for t in tasks}
     events = []
-    # line 2: update token footprint for t in T_act via turn probing
+    # refresh the footprints of the active tasks (turn probing)
     for tid, tokens in (new_footprints or {}).items():
         if by_id[tid].state == "active":
             by_id[tid].footprint = int(tokens)
-    # line 3: for each rank r
     for r, B in enumerate(budgets):
-        # lines 4-7: while TokenUsage(r) > B_r: preempt argmin Priority over the active tasks of r
+        # over budget: preempt the active task of this rank with the smallest Priority, one at a time
         while token_usage(tasks, r) > B:
             act = [t for t in tasks if t.state == "active" and t.rank == r]
             if not act:
@@ -90,7 +91,7 @@ def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_li
             t_evict = min(act, key=lambda t: (priority(t, tasks, w, ctx_norm), t.id))
             t_evict.state = "paused"
             events.append(("evict", t_evict.id, r))
-        # lines 8-18: while TokenUsage(r) < B_r
+        # headroom: resume before admitting, stop when neither is possible
         while token_usage(tasks, r) < B:
             usage = token_usage(tasks, r)
             paused_fit = [t for t in tasks if t.state == "paused" and t.rank in (-1, r) and usage + t.footprint <= B]
@@ -101,7 +102,7 @@ def schedule_pass(tasks, new_queue, budgets, w: Weights, ctx_norm: float, env_li
                 t_res.rank = r
                 events.append(("resume", t_res.id, r))
             else:
-                # line 13: admit a new task if it satisfies the constraints
+                # no paused task can run here: a new task, if the admission constraints allow one
                 in_flight = sum(1 for t in tasks if t.state in ("active", "paused")) + unconsumed
                 fits = [tid for tid in new_queue[:window] if usage + by_id[tid].probed <= B]
                 if fits and n_active < env_limit and (inflight_cap is None or in_flight < inflight_cap):

@@ -139,3 +139,120 @@ def test_staleness_and_diversity_constraints_match_the_listing():
     assert s.schedule() == []                                  # 2 active + 1 unconsumed = cap
     s.consume(1)
     assert [e[1] for e in s.schedule()] == [3]
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Direct pins of the oracle.  Every expected decision list below was worked out by hand from Algorithm 1 (preempt
+# the smallest Priority while over budget, then resume before admitting while under it) and the Priority sum of
+# Section 4.2 with weights 8 / 4 / 2 / 1 and L_context = tokens / 8192; neither implementation was consulted.
+W = oracle.Weights()
+CTX = 8192.0
+
+
+def _task(tid, group, fp, state="active", rank=0, is_eval=False, kind=0, probed=None):
+    return oracle.Task(tid, group, is_eval, fp if probed is None else probed, kind=kind, footprint=fp, state=state, rank=rank)
+
+
+def test_oracle_priority_is_the_weighted_sum_of_section_4_2():
+    tasks = [_task(0, 0, 3000, is_eval=True), _task(1, 1, 3000), _task(2, 2, 3000), _task(3, 1, 2000),
+             _task(4, 1, 500, state="done"), _task(5, 3, 16384, state="paused")]
+    want = {0: 8 + 0 + 2 + 3000 / 8192,            # evaluation task, alone in its group
+            1: 4 * (1 / 3) + 2 + 3000 / 8192,      # one of three group members has finished
+            2: 0 + 2 + 3000 / 8192,
+            3: 4 * (1 / 3) + 2 + 2000 / 8192,
+            5: 0 + 0 + 1.0}                        # paused: no active term; context factor capped at 1
+    for tid, p in want.items():
+        assert abs(oracle.priority(tasks[tid], tasks, W, CTX) - p) < 1e-12, tid
+
+
+def test_oracle_preempts_in_the_tier_order_of_table_1():
+    tasks = [_task(0, 0, 3000, is_eval=True), _task(1, 1, 3000), _task(2, 2, 3000), _task(3, 1, 2000),
+             _task(4, 1, 500, state="done")]
+    run = lambda B: oracle.schedule_pass(tasks, [], [B], W, CTX, env_limit=100)
+    # usage 11000: the task with no tier in its favour goes; nothing paused fits the 2000 tokens of headroom
+    assert run(10_000) == [("evict", 2, 0)]
+    # of the two members of the part-finished group the shorter context goes first
+    assert run(7_000) == [("evict", 3, 0)]
+    assert run(4_000) == [("evict", 1, 0)]
+    # the evaluation task is the last to go; with the rank empty the only paused task that fits 2500 comes back
+    assert run(2_500) == [("evict", 0, 0), ("resume", 3, 0)]
+    # headroom again: paused tasks return in Priority order (evaluation, then the part-finished group) while they fit
+    assert run(10_000) == [("resume", 0, 0), ("resume", 1, 0)]
+    assert [t.state for t in tasks] == ["active", "active", "paused", "active", "done"]
+    assert oracle.token_usage(tasks, 0) == 8000
+
+
+def test_oracle_affinity_resume_before_admit_and_footprint_refresh_on_two_ranks():
+    tasks = [_task(0, 0, 3000, rank=0), _task(1, 1, 3100, rank=0), _task(2, 2, 1000, rank=1),
+             _task(3, 3, 0, state="new", rank=-1, probed=2000), _task(4, 4, 0, state="new", rank=-1, probed=2500)]
+    queue = [3, 4]
+    # rank 0 holds 6100 > 5000: the shorter of its two equal-tier tasks is preempted and does not fit back (3100 + 3000).
+    # rank 1 has room for it (1000 + 3000) but the task may only return to rank 0, so rank 1 admits from the queue:
+    # task 3 (1000 + 2000), then task 4 no longer fits (3000 + 2500 > 5000)
+    ev = oracle.schedule_pass(tasks, queue, [5000, 5000], W, CTX, env_limit=100)
+    assert ev == [("evict", 0, 0), ("admit", 3, 1)]
+    assert queue == [4] and tasks[3].footprint == 2000 and tasks[0].rank == 0
+    # task 1 finishes; probing reports task 2 at 1800 tokens (and a number for the paused task 0, which must be ignored).
+    # rank 0 is empty: the paused task returns there BEFORE the queued task 4 is admitted beside it (3000 + 2500 > 5000: not at all)
+    tasks[1].state = "done"
+    ev = oracle.schedule_pass(tasks, queue, [5000, 5000], W, CTX, env_limit=100, new_footprints={2: 1800, 0: 9999})
+    assert ev == [("resume", 0, 0)]
+    assert tasks[2].footprint == 1800 and tasks[0].footprint == 3000
+    assert oracle.token_usage(tasks, 0) == 3000 and oracle.token_usage(tasks, 1) == 3800
+    # a larger budget on rank 0 lets the queued task in there, after the resume of the pass before
+    ev = oracle.schedule_pass(tasks, queue, [6000, 5000], W, CTX, env_limit=100)
+    assert ev == [("admit", 4, 0)] and queue == []
+
+
+def test_oracle_admission_constraints_by_hand():
+    # environment concurrency: two active tasks is the limit, so neither the paused task nor the queue moves
+    tasks = [_task(0, 0, 100), _task(1, 1, 100), _task(2, 2, 100, state="paused"), _task(3, 3, 0, state="new", rank=-1, probed=100)]
+    assert oracle.schedule_pass(tasks, [3], [10_000], W, CTX, env_limit=2) == []
+    assert oracle.schedule_pass(tasks, [3], [10_000], W, CTX, env_limit=3) == [("resume", 2, 0)]
+    # task diversity: the rank runs two tasks of type 0; of the queued types 0, 0, 1 the type-1 task goes first,
+    # then the others in arrival order (their type is the most common one either way)
+    tasks = [_task(0, 0, 100, kind=0), _task(1, 1, 100, kind=0)] + [
+        _task(i, i, 0, state="new", rank=-1, probed=100, kind=k) for i, k in ((2, 0), (3, 0), (4, 1))]
+    queue = [2, 3, 4]
+    assert oracle.schedule_pass(tasks, queue, [100_000], W, CTX, env_limit=100, window=3) == [
+        ("admit", 4, 0), ("admit", 2, 0), ("admit", 3, 0)]
+    # window 1 is plain arrival order
+    tasks = [_task(0, 0, 100, kind=0)] + [_task(i, i, 0, state="new", rank=-1, probed=100, kind=k) for i, k in ((1, 0), (2, 1))]
+    assert oracle.schedule_pass(tasks, [1, 2], [100_000], W, CTX, env_limit=100, window=1) == [("admit", 1, 0), ("admit", 2, 0)]
+    # policy staleness: cap 3 counts active + paused + finished-but-unconsumed trajectories
+    tasks = [_task(i, i, 0, state="new", rank=-1, probed=100) for i in range(5)]
+    queue = [0, 1, 2, 3, 4]
+    kw = dict(budgets=[100_000], w=W, ctx_norm=CTX, env_limit=100, inflight_cap=3)
+    assert oracle.schedule_pass(tasks, queue, unconsumed=0, **kw) == [("admit", 0, 0), ("admit", 1, 0), ("admit", 2, 0)]
+    tasks[0].state = "done"
+    assert oracle.schedule_pass(tasks, queue, unconsumed=1, **kw) == []            # 2 active + 1 unconsumed = cap
+    assert oracle.schedule_pass(tasks, queue, unconsumed=0, **kw) == [("admit", 3, 0)]
+
+
+def test_oracle_pass_invariants_on_random_states():
+    """What the loop guarantees whatever the readings: a rank ends a pass over budget only when one task alone is
+    too large for it (or nothing is left to preempt), every resume on a rank precedes every admit there, and a
+    paused task comes back only to the rank it left."""
+    rng = np.random.default_rng(7)
+    for trial in range(200):
+        n_ranks = int(rng.integers(1, 4))
+        budgets = [int(rng.integers(1000, 6000)) for _ in range(n_ranks)]
+        tasks, queue = [], []
+        for tid in range(int(rng.integers(3, 14))):
+            state = ["active", "paused", "new", "done"][int(rng.integers(0, 4))]
+            fp = int(rng.integers(100, 3000))
+            rank = int(rng.integers(0, n_ranks)) if state in ("active", "paused") else -1
+            tasks.append(_task(tid, int(rng.integers(0, 4)), fp if state != "new" else 0, state=state, rank=rank,
+                               is_eval=bool(rng.random() < 0.2), probed=fp))
+            if state == "new":
+                queue.append(tid)
+        home = {t.id: t.rank for t in tasks if t.state == "paused"}
+        ev = oracle.schedule_pass(tasks, queue, budgets, W, CTX, env_limit=int(rng.integers(1, 12)))
+        for r, B in enumerate(budgets):
+            act = [t for t in tasks if t.state == "active" and t.rank == r]
+            assert oracle.token_usage(tasks, r) <= B or len(act) <= 1
+            kinds_r = [k for k, _, rr in ev if rr == r and k != "evict"]
+            assert kinds_r == sorted(kinds_r, key=lambda k: k != "resume"), "an admit came before a resume"
+        for k, tid, r in ev:
+            if k == "resume" and tid in home:
+                assert home[tid] == r

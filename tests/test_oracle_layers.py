@@ -99,3 +99,39 @@ def test_prune_refuses_without_changing_anything_hand_traced():
     c.release(0)
     c.prune(1, 2, 4)
     assert list(c.page_table(1)) == [0, 1, 2, 3] and c.task_len(1) == 14 and c.free_pages() == 0
+
+
+def test_reset_of_the_layered_oracle_flushes_every_layer_alike():
+    """After a reset every layer hands pages out in the new order, holds no task, and keeps layers apart as before:
+    checked against per-layer token lists that are simply emptied."""
+    rng = np.random.default_rng(5)
+    L, S, HKV, D, P = 3, 4, 1, 4, 8
+    orc = LayeredKVOracle(L, num_pages=P, page_size=S, num_kv_heads=HKV, head_dim=D, max_tasks=4, max_pages_per_task=8,
+                          free_order=[7, 6, 5, 4, 3, 2, 1, 0])
+    orc.alloc(0)
+    orc.alloc(1)
+    orc.append([0, 1], [0, 6, 9], np.stack([_rows(rng, 9, HKV, D) for _ in range(L)]), np.stack([_rows(rng, 9, HKV, D) for _ in range(L)]))
+    assert list(orc.page_table(0)) == [7, 6] and list(orc.page_table(1)) == [5]
+    orc.fork(0, 2)
+    orc.reset([1, 3, 5, 7, 0, 2, 4, 6])
+    assert orc.free_pages() == P and orc.used_tokens() == 0
+    for l in range(L):
+        assert orc.layer(l).live == {} and orc.layer(l).ref == {}
+        assert orc.layer(l).free_stack_top_first() == [1, 3, 5, 7, 0, 2, 4, 6]
+    with pytest.raises(OracleError):
+        orc.task_len(0)
+    orc.alloc(2)
+    nk = np.stack([_rows(rng, 5, HKV, D) for _ in range(L)])
+    nv = np.stack([_rows(rng, 5, HKV, D) for _ in range(L)])
+    orc.append([2], [0, 5], nk, nv)
+    assert list(orc.page_table(2)) == [1, 3]
+    for l in range(L):
+        k, v = orc.read(l, 2)
+        assert np.array_equal(k, nk[l]) and np.array_equal(v, nv[l])       # layer l holds layer l's rows, nothing older
+    orc.reset(None)
+    orc.alloc(0)
+    orc.append([0], [0, 1], nk[:, :1], nv[:, :1])
+    assert list(orc.page_table(0)) == [0]
+    with pytest.raises(OracleError):
+        orc.reset([0, 0, 1, 2, 3, 4, 5, 6])
+    assert orc.task_len(0) == 1 and orc.free_pages() == P - 1

@@ -348,3 +348,55 @@ def test_refcount_conservation_under_random_ops_with_forks():
         assert kk.shape[0] == len(shadow[t])
         for pos, row in enumerate(shadow[t]):
             assert np.array_equal(kk[pos], row)
+
+
+def test_reset_flushes_everything_and_primes_the_stack_in_the_given_order():
+    """Hand trace on the 6-page pool (page size 4): after a reset the pool behaves like a fresh one created with
+    that order - pages come out as order[0], order[1], ... - whatever was resident before (the flush that follows
+    a weight synchronisation, Section 5.2)."""
+    def rows(n):
+        k = np.arange(n * 2, dtype=np.uint16).reshape(n, 1, 2)
+        return k, k + np.uint16(9)
+
+    c = PagedKVOracle(6, 4, 1, 2, max_tasks=4, max_pages_per_task=6, free_order=[3, 0, 5, 1, 4, 2])
+    for t in (0, 1):
+        c.alloc(t)
+    c.append([0, 1], [0, 9, 14], *rows(14))                  # 3 + 2 pages: [3, 0, 5] and [1, 4]
+    c.fork(1, 2)                                             # shares page 1, copies the partial page 4 into page 2
+    assert c.free_pages() == 0 and list(c.page_table(2)) == [1, 2]
+    c.reset([2, 4, 0, 5, 1, 3])
+    assert c.free_pages() == 6 and c.used_tokens() == 0 and c.ref == {} and c.live == {}
+    assert c.free_stack_top_first() == [2, 4, 0, 5, 1, 3]
+    for t in (0, 1, 2):
+        with pytest.raises(OracleError) as e:                # every task is unknown afterwards
+            c.task_len(t)
+        assert e.value.code == pk.ERR_UNKNOWN_TASK
+    c.alloc(1)
+    c.alloc(0)
+    c.append([1], [0, 5], *rows(5))
+    assert list(c.page_table(1)) == [2, 4]
+    c.append([0, 1], [0, 1, 5], *rows(5))                    # task 0 takes the next page, task 1 fills page 4 and takes one more
+    assert list(c.page_table(0)) == [0] and list(c.page_table(1)) == [2, 4, 5]
+    assert c.free_stack_top_first() == [1, 3]
+    # same content as a fresh pool created with that order and given the same calls
+    f = PagedKVOracle(6, 4, 1, 2, max_tasks=4, max_pages_per_task=6, free_order=[2, 4, 0, 5, 1, 3])
+    f.alloc(1)
+    f.alloc(0)
+    f.append([1], [0, 5], *rows(5))
+    f.append([0, 1], [0, 1, 5], *rows(5))
+    assert f.state_hash() == c.state_hash()
+    for t in (0, 1):
+        assert all(np.array_equal(a, b) for a, b in zip(c.read(t), f.read(t)))
+    # no order = identity: pages 0, 1, 2, ...
+    c.reset()
+    assert c.free_stack_top_first() == [0, 1, 2, 3, 4, 5]
+    c.alloc(3)
+    c.append([3], [0, 9], *rows(9))
+    assert list(c.page_table(3)) == [0, 1, 2]
+    # an order that is not a permutation is refused and changes nothing
+    before = c.state_hash()
+    for bad in ([0, 1, 2, 3, 4, 4], [0, 1, 2, 3, 4], [0, 1, 2, 3, 4, 6]):
+        with pytest.raises(OracleError) as e:
+            c.reset(bad)
+        assert e.value.code == pk.ERR_INVALID_ARG
+        assert c.state_hash() == before and c.task_len(3) == 9
