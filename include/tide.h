@@ -215,7 +215,14 @@ int tide_kv_read(tide_kv_t* kv, int32_t layer, int32_t task, void* out_k /*devic
                  void* stream);
 
 /* Synchronises `stream` and returns the device status word: TIDE_OK, or TIDE_ERR_DEVICE_TIMEOUT if a
- * bounded wait in a kernel ran out since the last call (the word is then cleared). */
+ * bounded wait in a kernel ran out since the last call (the word is then cleared).  Every wait inside the
+ * attention kernels (for a K/V stage, a tensor-core result, a free buffer) has a time limit; when one runs out
+ * the thread block records the time-out, finishes without waiting again and frees what it holds, and the kernel
+ * returns by itself.  The word is sticky: from the time-out until this call clears it, thread blocks of that
+ * launch and of every later attention launch on the handle leave without computing, so `out` / `lse` of those
+ * calls are undefined although the calls themselves returned TIDE_OK.  A caller that needs to know asks
+ * tide_status after the step; after a TIDE_ERR_DEVICE_TIMEOUT the cache contents are intact and the attention
+ * call can simply be repeated. */
 int tide_status(tide_kv_t* kv, void* stream);
 
 /* Rows of the most recently planned batch (tide_attend, tide_step_begin) that were planned as groups sharing their
@@ -230,6 +237,25 @@ int tide_last_sharing(tide_kv_t* kv, int64_t* groups, int64_t* rows);
  * tensor-tile paths, rows merged, and kernels launched by the most recent append + attend pair. */
 int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items, int64_t* merge_rows,
                    int64_t* kernel_launches);
+
+/* Planner settings and test hooks of one handle.  The defaults are the measured best on B200; nothing reads the
+ * environment.  Changing a setting closes an open step (tide_step_begin must be called again).
+ * TIDE_ERR_INVALID_ARG for an unknown knob or a value outside its range. */
+typedef enum {
+  TIDE_TUNE_ITEMS_PER_SM = 0,     /* work items per SM the KV-split planner aims for, 1..64 (default 3)            */
+  TIDE_TUNE_GROUPING = 1,         /* 0: never plan forked rows as groups that read shared pages once (default 1)   */
+  TIDE_TUNE_MIN_SAVED_BYTES = 2,  /* KV bytes a batch must save before groups are used (default 64 MiB)            */
+  TIDE_TUNE_HOST_STEP_CHUNKS = 3, /* row groups of tide_step_host, 1..8; 0 = chosen by transfer size (default)     */
+  TIDE_TUNE_UMMA_MIN_ROWS = 4,    /* packed rows (q_len * Hq/Hkv) from which a head_dim-128 row runs on the        */
+                                  /* tcgen05 kernel, >= 17 (default 17)                                            */
+  TIDE_TUNE_WAIT_LIMIT_US = 5,    /* time limit of every wait inside a kernel, microseconds (default 2 000 000)    */
+  TIDE_TUNE_DROP_FIRST_STAGE = 6  /* test hook, non-zero arms it for the NEXT attention call only: in work item 0   */
+                                  /* of each attention kernel of that call the K/V producer leaves out (its part   */
+                                  /* of) the first stage, so the wait for that stage runs out and the time-out     */
+                                  /* path of tide_status can be exercised without any fault.  Results of that      */
+                                  /* call are undefined.                                                           */
+} tide_tune_t;
+int tide_tune(tide_kv_t* kv, int knob, int64_t value);
 
 /* Per-phase device timing of the calls that follow (CUDA events on the caller's stream; off by default).
  * tide_phase_ms waits for the most recent tide_attend and returns the milliseconds spent in the most
@@ -251,9 +277,12 @@ int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile
  * table, on layer 0.  Limits: at most TIDE_STATIC_MAX_ROWS rows per call (more returns TIDE_ERR_WORKSPACE), decode-style
  * rows only (others return TIDE_ERR_INVALID_ARG); long rows are split over KV only as far as the fixed array
  * allows.  The first call on a device looks up the array's device address; make that call before any stream
- * capture begins.  Every call uses the same array and overwrites what the previous call left there (nothing in
- * it needs clearing between calls), so two calls whose kernels may overlap on the GPU (different streams) race:
- * keep the calls of one process on one stream, or order them with events. */
+ * capture begins.  The device the handle was created on must be current (TIDE_ERR_INVALID_ARG otherwise).  The
+ * call copies nothing from host memory: the row records travel as kernel arguments and are expanded on the
+ * device, so it is asynchronous on `stream`.  Every call uses the same array and overwrites what the previous
+ * call left there (every record a call reads it has written itself, so nothing needs clearing between calls),
+ * and two calls whose kernels may overlap on the GPU (different streams) race: keep the calls of one process on
+ * one stream, or order them with events. */
 #define TIDE_STATIC_MAX_ROWS 64
 int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows /*host*/,
                               const void* q /*device*/, float scale, void* out /*device*/,

@@ -42,7 +42,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(HERE, "build", os.path.basename(src) + ".o")
         cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
                "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v" if verbose else "-O3",
-               "-c", src, "-o", obj] + (["-DTIDE_UMMA_TIMING"] if os.environ.get("TIDE_UMMA_TIMING") else []) + os.environ.get("TIDE_EXTRA_NVCC", "").split()
+               "-c", src, "-o", obj]
         procs.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False

@@ -89,7 +89,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
     return;
   }
 
-  // a bounded wait that ran out in an earlier CTA of this launch means something is wrong: start no more work
+  // The status word is set when a bounded wait runs out and stays set until tide_status clears it.  While it is
+  // set no CTA starts work (this launch's later CTAs and every CTA of later launches leave here without writing
+  // anything), so outputs are undefined from the time-out until the caller has read the status.
   __shared__ int s_skip;
   if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int*>(P.status);
   __syncthreads();
@@ -111,9 +113,13 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
   if (warp == kConsumerWarps) {
     // ================= producer warp =================
     const int pages_per_stage = kStageKeys / g.S;
+    int issued = 0;                              // stages whose copies were issued
     for (int st = 0; st < n_st; ++st) {
       const int slot = st % kStages;
-      if (st >= kStages) mbar_wait(smem_u32(&s_empty[slot]), ((st / kStages) - 1) & 1, abort_flag, P.status);
+      // a wait that gave up means the ring can no longer be trusted: issue nothing more
+      if (st >= kStages && !mbar_wait(smem_u32(&s_empty[slot]), ((st / kStages) - 1) & 1, abort_flag, P.status, P.wait_limit_ns)) break;
+      issued = st + 1;
+      if (P.debug_drop_first_stage != 0 && item == 0 && st == 0) continue;   // test hook: this stage never arrives
       const int key0 = kv_begin + st * kStageKeys;
       const int npages = min(pages_per_stage, (kv_end - key0 + g.S - 1) / g.S);
       const uint32_t bar = smem_u32(&s_full[slot]);
@@ -126,11 +132,13 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
       }
     }
     if (*abort_flag && lane == 0) {
-      // a wait gave up somewhere: do not leave the CTA while copies into its shared memory are in flight
-      for (int st = max(0, n_st - kStages); st < n_st; ++st) {
+      // a wait gave up somewhere: do not leave the CTA while copies into its shared memory are in flight.  Only the
+      // last kStages stages that were issued can still be landing (an older one was consumed before its slot was
+      // refilled); each wait is bounded like every other.
+      for (int st = max(0, issued - kStages); st < issued; ++st) {
         const uint32_t bar = smem_u32(&s_full[st % kStages]);
         const long long t0 = global_ns();
-        while (!mbar_try(bar, (st / kStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try(bar, (st / kStages) & 1) && global_ns() - t0 < P.wait_limit_ns) {}
       }
     }
     return;
@@ -171,7 +179,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
 
   for (int st = 0; st < n_st; ++st) {
     const int slot = st % kStages;
-    mbar_wait(smem_u32(&s_full[slot]), (st / kStages) & 1, abort_flag, P.status);
+    mbar_wait(smem_u32(&s_full[slot]), (st / kStages) & 1, abort_flag, P.status, P.wait_limit_ns);
     const int key0 = kv_begin + st * kStageKeys;
     const uint32_t stage = smem_base + slot * STAGE_BYTES;
     const int kb_first = DECODE ? warp : 0;

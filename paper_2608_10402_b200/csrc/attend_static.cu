@@ -9,7 +9,11 @@
 // array below, which every GPU that loads the library holds until the process exits.
 //
 // The array's name is only a host-side stand-in in host code; the device address is looked up once per device
-// with cudaGetSymbolAddress and handed to the (unchanged) decode and merge kernels.
+// with cudaGetSymbolAddress and handed to the (unchanged) decode and merge kernels.  The row descriptors reach
+// the device as kernel arguments of a small set-up kernel that expands them into the array, so the call makes no
+// copy from host memory at all and is asynchronous on its stream.
+#include <atomic>
+
 #include "tide_internal.h"
 
 using namespace tide;
@@ -27,16 +31,64 @@ constexpr size_t kScratchBytes = kPartOff + (size_t)kMaxPartRows * kMaxD * sizeo
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_ptr[kMaxDevices];             // device address of the array, per device
-bool g_scratch_ready[kMaxDevices];
+// Device address of the array, per device.  The lookup gives the same answer every time, so threads that race
+// on the first call of a device all store the same value.
+std::atomic<unsigned char*> g_scratch_ptr[kMaxDevices];
 
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// One row as the host planned it; the set-up kernel turns these into Segment records.
+struct StaticRow {
+  int32_t table_off, n, p, n_splits, chunk;
+};
+struct StaticPlanArgs {          // passed by value (about 1.3 KB of kernel arguments)
+  int32_t n_rows, Hkv, Hq;
+  StaticRow rows[kMaxRows];
+};
+
+// Expands the planned rows into the decode list (segs[0 .. n_rows)) and the merge list (segs[kMaxRows ...)): the
+// running sums over rows (query offset, first work item, first partial row, first merge row) are taken here, by
+// one thread, in row order - at most 64 rows.  Every field of every record written is set, so nothing of an
+// earlier call's records shows through.
+__global__ void static_plan_kernel(const StaticPlanArgs a, Segment* __restrict__ segs) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  int qoff = 0, items = 0, part = 0, merge = 0, n_merge = 0;
+  for (int b = 0; b < a.n_rows; ++b) {
+    const StaticRow r = a.rows[b];
+    Segment s;
+    s.table_off = r.table_off;
+    s.q_off = qoff;
+    s.n = r.n;
+    s.p = r.p;
+    s.item_base = items;
+    s.n_mtiles = 1;
+    s.n_splits = r.n_splits;
+    s.chunk = r.chunk;
+    s.part_base = 0;
+    s.merge_base = 0;
+    s.causal = 1;
+    s.origin = 0;
+    s.partial = 0;
+    s.x_part_base = 0;
+    s.x_n_splits = 0;
+    s.x_stride = 0;
+    items += a.Hkv * r.n_splits;
+    if (r.n_splits > 1) {
+      s.part_base = part;
+      s.merge_base = merge;
+      part += r.n_splits * r.n * a.Hq;
+      merge += r.n * a.Hq;
+      segs[kMaxRows + n_merge++] = s;
+    }
+    segs[b] = s;
+    qoff += r.n;
+  }
+}
+
 }  // namespace
 
-// Defined in tide_host.cu; narrow accessors so that this file needs nothing else of the handle.
-extern "C" int tide_internal_view(tide_kv_t* kv, Geom* g, const uint8_t** pool, const int32_t** table, int** status,
-                                  const int32_t** len, const uint8_t** live, int32_t* max_tasks);
+// Defined in tide_host.cu; a narrow accessor so that this file needs nothing else of the handle.
+extern "C" int tide_internal_view(tide_kv_t* kv, tide::StaticView* v);
 
 extern "C" int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, const void* q,
                                          float scale, void* out, float* lse, void* stream) {
@@ -46,44 +98,47 @@ extern "C" int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const ti
   if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)lse & 3) || !(scale == scale)) return TIDE_ERR_INVALID_ARG;
   if (n_rows > kMaxRows) return TIDE_ERR_WORKSPACE;      // beyond the fixed scratch: use tide_attend
 
-  Geom g;
-  const uint8_t* pool; const int32_t* table; int* status; const int32_t* len; const uint8_t* live; int32_t max_tasks;
-  int rc = tide_internal_view(kv, &g, &pool, &table, &status, &len, &live, &max_tasks);
+  StaticView v;
+  int rc = tide_internal_view(kv, &v);
   if (rc != TIDE_OK) return rc;
+  const Geom& g = v.g;
   if (g.D > kMaxD) return TIDE_ERR_WORKSPACE;
-  long long total_q = 0;
   for (int b = 0; b < n_rows; ++b) {
     const tide_row_t& r = rows[b];
-    if (r.task < 0 || r.task >= max_tasks) return TIDE_ERR_INVALID_ARG;
-    if (!live[r.task]) return TIDE_ERR_UNKNOWN_TASK;
-    if (!(r.q_len >= 1 && r.q_len <= r.ctx_len && r.ctx_len <= len[r.task])) return TIDE_ERR_CTX_RANGE;
-    if (r.q_len * g.G > kDecodeTileRows) return TIDE_ERR_INVALID_ARG;   // decode-style rows only
-    total_q += r.q_len;
+    if (r.task < 0 || r.task >= v.max_tasks) return TIDE_ERR_INVALID_ARG;
+    if (!v.live[r.task]) return TIDE_ERR_UNKNOWN_TASK;
+    if (!(r.q_len >= 1 && r.q_len <= r.ctx_len && r.ctx_len <= v.len[r.task])) return TIDE_ERR_CTX_RANGE;
+    if (r.q_len > kDecodeTileRows / g.G) return TIDE_ERR_INVALID_ARG;   // decode-style rows only
   }
 
   // ---- once per device: the device address of the scratch array (first call; do it before any capture) ----
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return TIDE_ERR_CUDA;
+  if (dev != v.device) return TIDE_ERR_INVALID_ARG;       // the handle's device must be current
   if (dev < 0 || dev >= kMaxDevices) return TIDE_ERR_WORKSPACE;
-  if (!g_scratch_ready[dev]) {
+  unsigned char* scratch = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (scratch == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return TIDE_ERR_CUDA;
-    g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
-    g_scratch_ready[dev] = true;
+    scratch = static_cast<unsigned char*>(p);
+    g_scratch_ptr[dev].store(scratch, std::memory_order_release);
   }
-  unsigned char* scratch = g_scratch_ptr[dev];
 
-  // ---- plan with fixed-size host arrays: split long rows over KV until the SMs are covered or the fixed
-  //      number of partial rows is used up ----
-  Segment segs[2 * kMaxRows];
+  // ---- plan: split long rows over KV towards the library's number of work items per SM, as far as the fixed
+  //      number of partial rows allows ----
+  StaticPlanArgs pa;
+  pa.n_rows = n_rows;
+  pa.Hkv = g.Hkv;
+  pa.Hq = g.Hq;
   long long w = 0;
   for (int b = 0; b < n_rows; ++b) w += (long long)g.Hkv * rows[b].ctx_len;
-  long long chunk_target = w / (148 * 8) + 1;
+  long long chunk_target = w / ((long long)v.num_sms * v.items_per_sm) + 1;
   if (chunk_target < 256) chunk_target = 256;
-  long long part_rows = 0;
+  long long items = 0, merge_rows = 0;
   for (int attempt = 0; attempt < 40; ++attempt) {
-    part_rows = 0;
-    long long qoff = 0;
+    long long part_rows = 0;
+    items = 0;
+    merge_rows = 0;
     for (int b = 0; b < n_rows; ++b) {
       const tide_row_t& r = rows[b];
       int n_splits = (int)((r.ctx_len + chunk_target - 1) / chunk_target);
@@ -91,45 +146,34 @@ extern "C" int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const ti
       if (n_splits < 1) n_splits = 1;
       const int chunk = ceil_div(ceil_div(r.ctx_len, n_splits), 2 * kStageKeys) * 2 * kStageKeys;
       n_splits = ceil_div(r.ctx_len, chunk);
-      Segment s{};
+      StaticRow& s = pa.rows[b];
       s.table_off = r.task * g.max_pages_per_task;
-      s.q_off = (int32_t)qoff;
       s.n = r.q_len;
       s.p = r.ctx_len - r.q_len;
-      s.n_mtiles = 1;
       s.n_splits = n_splits;
       s.chunk = chunk;
-      s.causal = 1;
-      if (n_splits > 1) part_rows += (long long)n_splits * r.q_len * g.Hq;
-      segs[b] = s;
-      qoff += r.q_len;
+      items += (long long)g.Hkv * n_splits;
+      if (n_splits > 1) {
+        part_rows += (long long)n_splits * r.q_len * g.Hq;
+        merge_rows += (long long)r.q_len * g.Hq;
+      }
     }
     if (part_rows <= kMaxPartRows) break;
     chunk_target *= 2;
     if (attempt == 39) return TIDE_ERR_WORKSPACE;
   }
-  long long items = 0, part_cursor = 0, merge_rows = 0;
   int n_merge = 0;
-  for (int b = 0; b < n_rows; ++b) {
-    Segment& s = segs[b];
-    s.item_base = (int32_t)items;
-    items += (long long)g.Hkv * s.n_splits;
-    if (s.n_splits > 1) {
-      s.part_base = (int32_t)part_cursor;
-      part_cursor += (long long)s.n_splits * s.n * g.Hq;
-      s.merge_base = (int32_t)merge_rows;
-      merge_rows += (long long)s.n * g.Hq;
-      segs[kMaxRows + n_merge++] = s;
-    }
-  }
+  for (int b = 0; b < n_rows; ++b) n_merge += pa.rows[b].n_splits > 1 ? 1 : 0;
 
-  // ---- descriptors into the scratch array (a plain copy from this stack frame), then the two kernels ----
+  // ---- the row records into the scratch array (kernel arguments, expanded on the device), then the two kernels ----
   cudaStream_t st = (cudaStream_t)stream;
-  if (cudaMemcpyAsync(scratch, segs, kSegBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return TIDE_ERR_CUDA;
+  Segment* d_segs = reinterpret_cast<Segment*>(scratch);
+  static_plan_kernel<<<1, 32, 0, st>>>(pa, d_segs);
+  if (cudaGetLastError() != cudaSuccess) return TIDE_ERR_CUDA;
   AttendParams ap;
-  ap.pool = pool;
-  ap.table = table;
-  ap.segs = reinterpret_cast<const Segment*>(scratch);
+  ap.pool = v.pool;
+  ap.table = v.table;
+  ap.segs = d_segs;
   ap.n_segs = n_rows;
   ap.n_items = (int)items;
   ap.q = (const uint16_t*)q;
@@ -138,12 +182,13 @@ extern "C" int tide_attend_decode_static(tide_kv_t* kv, int32_t n_rows, const ti
   ap.part_lse = reinterpret_cast<float*>(scratch + kLseOff);
   ap.part_o = reinterpret_cast<float*>(scratch + kPartOff);
   ap.scale_log2e = scale * 1.4426950408889634f;
-  ap.status = status;
+  ap.status = v.status;
   ap.g = g;
+  ap.wait_limit_ns = v.wait_limit_ns;
   if (launch_attend_decode(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
   if (merge_rows > 0) {
     MergeParams mp;
-    mp.segs = reinterpret_cast<const Segment*>(scratch) + kMaxRows;
+    mp.segs = d_segs + kMaxRows;
     mp.n_segs = n_merge;
     mp.n_rows = (int)merge_rows;
     mp.part_o = ap.part_o;

@@ -141,36 +141,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Optional cycle accounting (compile with -DTIDE_UMMA_TIMING): where the softmax warps and the MMA lane
-// spend their time, accumulated into 64-bit counters behind the status word.
-#ifdef TIDE_UMMA_TIMING
-#define TT_DECL long long tt_wait = 0, tt_wait2 = 0, tt_t0 = clock64(), tt_a
-#define TT_BEGIN tt_a = clock64()
-#define TT_END(acc) acc += clock64() - tt_a
-#define TT_FLUSH(i0, i1, i2)                                                                       \
-  do {                                                                                              \
-    unsigned long long* c = reinterpret_cast<unsigned long long*>(P.status) + 8;                   \
-    atomicAdd(c + (i0), (unsigned long long)tt_wait);                                               \
-    atomicAdd(c + (i1), (unsigned long long)tt_wait2);                                              \
-    atomicAdd(c + (i2), (unsigned long long)(clock64() - tt_t0));                                   \
-  } while (0)
-// per-phase accounting: TT_PH(i) adds the cycles since the previous mark to phase i
-#define TT_PH_DECL long long tt_ph[6] = {0, 0, 0, 0, 0, 0}, tt_b = 0
-#define TT_PH_START tt_b = clock64()
-#define TT_PH(i) do { const long long now_ = clock64(); tt_ph[i] += now_ - tt_b; tt_b = now_; } while (0)
-#define TT_PH_FLUSH(i0) do { unsigned long long* c = reinterpret_cast<unsigned long long*>(P.status) + 8; \
-    for (int i_ = 0; i_ < 6; ++i_) atomicAdd(c + (i0) + i_, (unsigned long long)tt_ph[i_]); } while (0)
-#else
-#define TT_PH_DECL
-#define TT_PH_START
-#define TT_PH(i)
-#define TT_PH_FLUSH(i0)
-#define TT_DECL
-#define TT_BEGIN
-#define TT_END(acc)
-#define TT_FLUSH(i0, i1, i2)
-#endif
-
 struct Bars {
   uint64_t kv_full[kNumBuf];
   uint64_t kv_empty[kNumBuf];
@@ -178,6 +148,7 @@ struct Bars {
   uint64_t s_full[2];   // S_t(j) is in TMEM (and every earlier MMA, PV_t(j-1) included, has retired)
   uint64_t p_full[2];   // P_t(j) is in TMEM
   uint64_t o_full[2];   // the last PV_t has retired
+  uint64_t mma_done;    // every MMA of the item has retired
 };
 
 __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendParams P) {
@@ -226,7 +197,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   const int n_tiles = max(t_tiles[0], t_tiles[1]);
   const int kv_end = max(t_end[0], t_end[1]);
 
-  // a bounded wait that ran out in an earlier CTA of this launch means something is wrong: start no more work
+  // The status word is set when a bounded wait runs out and stays set until tide_status clears it; while it is set
+  // no CTA starts work, so outputs are undefined from the time-out until the caller has read the status.
   __shared__ int s_skip;
   if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int*>(P.status);
   __syncthreads();
@@ -241,6 +213,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
       mbar_init(smem_u32(&bars.p_full[t]), 128);
       mbar_init(smem_u32(&bars.o_full[t]), 1);
     }
+    mbar_init(smem_u32(&bars.mma_done), 1);
     mbar_fence_init();
   }
   if (warp == 9) {
@@ -278,11 +251,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           return lp < g.max_pages_per_task ? trow[lp] : 0;
         };
         int ids_cur = load_ids(0), ids_nxt = load_ids(1), cur_grp = 0;
+        int issued = 0;                                        // tiles this warp has issued its copies of
         for (int j = 0; j < n_tiles; ++j) {
           const int buf = j % kNumBuf, use = j / kNumBuf;
           const int grp = j / tiles_per_group;
           if (grp != cur_grp) { ids_cur = ids_nxt; ids_nxt = load_ids(grp + 1); cur_grp = grp; }
-          if (use > 0) mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status);
+          // a wait that gave up means the ring can no longer be trusted: issue nothing more
+          if (use > 0 && !mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status, P.wait_limit_ns)) break;
+          issued = j + 1;
+          if (P.debug_drop_first_stage != 0 && item == 0 && j == 0 && pw == 0) continue;   // test hook: this warp's part of tile 0 never arrives
           const int key0 = kv_begin + j * kTileKeys;
           const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
           const uint32_t bar = smem_u32(&bars.kv_full[buf]);
@@ -299,21 +276,22 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
             bulk_g2s(smem_base + buf * kSlotBytes + is_v * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
           }
         }
-        if (*abort_flag && lane == 0 && pw == 0) {
-          // a wait gave up somewhere: do not leave while copies into this CTA's shared memory are in flight
-          for (int idx = max(0, n_tiles - kNumBuf); idx < n_tiles; ++idx) {
+        if (*abort_flag && lane == 0) {
+          // a wait gave up somewhere: this warp does not leave while copies it issued into the CTA's shared memory
+          // can still be landing.  Those are among its last kNumBuf tiles (an older one was consumed before its slot
+          // was refilled); a tile's barrier completes when all three producer warps' parts are in, and each wait is
+          // bounded like every other (a tile another warp never issued its part of runs into that bound).
+          for (int idx = max(0, issued - kNumBuf); idx < issued; ++idx) {
             const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
             const long long t0 = global_ns();
-            while (!mbar_try(bar, (idx / kNumBuf) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+            while (!mbar_try(bar, (idx / kNumBuf) & 1) && global_ns() - t0 < P.wait_limit_ns) {}
           }
         }
       }
     } else if (warp == 9) {
       // ================= MMA issuer (whole warp converged, one elected lane issues) =================
       if (n_tiles > 0) {
-        TT_DECL;
-        TT_PH_DECL;
-        mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status);
+        mbar_wait(smem_u32(&bars.q_full), 0, abort_flag, P.status, P.wait_limit_ns);
         tc_fence_after();
         auto issue_qk = [&](int t, int j) {
           const uint32_t kbuf = smem_base + (j % kNumBuf) * kSlotBytes;
@@ -331,9 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
                    (j > 0 || ks > 0) ? 1u : 0u);
         };
         auto wait_full = [&](int idx) {
-          TT_BEGIN;
-          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
-          TT_END(tt_wait2);
+          mbar_wait(smem_u32(&bars.kv_full[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status, P.wait_limit_ns);
         };
         wait_full(0);
         tc_fence_after();
@@ -352,38 +328,29 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
             __syncwarp();
           }
           bool k_ready = false;
-          TT_PH_START;
           for (int t = 0; t < 2; ++t) {
             if (j < t_tiles[t]) {
-              TT_BEGIN;
-              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status);
-              TT_END(tt_wait);
-              TT_PH(0);
+              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status, P.wait_limit_ns);
               tc_fence_after();
-              TT_PH(1);
               issue_pv(t, j);
-              TT_PH(2);
               if (j + 1 < t_tiles[t]) {
                 if (!k_ready) { wait_full(j + 1); k_ready = true; }
-                TT_PH(3);
                 issue_qk(t, j + 1);                          // overwrites S_t / P_t after PV_t(j), in order
-                TT_PH(4);
               } else {
                 mma_commit(smem_u32(&bars.o_full[t]));
               }
             }
           }
           mma_commit(smem_u32(&bars.kv_empty[j % kNumBuf]));   // K_j and V_j are consumed once PV(j) retires
-          TT_PH(5);
         }
-        // every MMA has completed (commits arrive in issue order) before this thread leaves
+        // Every MMA has retired before this warp leaves (TMEM is freed after the CTA's last barrier): one more commit
+        // covers all of them.  This wait does not look at the abort flag - MMAs retire whatever else went wrong.
+        mma_commit(smem_u32(&bars.mma_done));
         {
-          const int idx = n_tiles - 1;
-          mbar_wait(smem_u32(&bars.kv_empty[idx % kNumBuf]), (idx / kNumBuf) & 1, abort_flag, P.status);
+          const uint32_t bar = smem_u32(&bars.mma_done);
+          const long long t0 = global_ns();
+          while (!mbar_try(bar, 0) && global_ns() - t0 < P.wait_limit_ns) {}
         }
-#ifdef TIDE_UMMA_TIMING
-        if (lane == 0) { TT_FLUSH(2, 3, 4); TT_PH_FLUSH(12); }   // counters 12..17: wait P, fence, PV, wait K/V, QK, commits
-#endif
       }
     }
   } else {
@@ -421,23 +388,17 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     const uint32_t s_addr = tmem + lane_addr + kColS + t * 64;
     const uint32_t o_addr = tmem + lane_addr + kColO + t * 128;
 
-    TT_DECL;
-    TT_PH_DECL;
     // One key tile of this row tile.  The tiles that need the causal (or end-of-range) mask are the last ones of the
     // item; they get a copy of the body of their own, so the 128 compare-and-select instructions of the mask are
     // not part of the code that the other ~99 % of the tiles run (its mere presence in the loop cost 2 %).
     auto tile = [&](const int j, auto masked_tag) {
       constexpr bool kMasked = decltype(masked_tag)::value;
-      TT_BEGIN;
-      mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status);
-      TT_END(tt_wait);
-      TT_PH_START;
+      mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag, P.status, P.wait_limit_ns);
       tc_fence_after();
       float s[64];
       tmem_ld32(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
       tmem_ld32(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_wait_ld();
-      TT_PH(0);
       if constexpr (kMasked) {
         const int vis = limit - (kv_begin + j * kTileKeys);
 #pragma unroll
@@ -475,7 +436,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
         }
       }
       m = m_new;
-      TT_PH(1);
       const float mu = (m == -INFINITY) ? 0.f : m;
       float sp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
@@ -498,13 +458,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 #pragma unroll
         for (int i = 0; i < 4; ++i) unpack2(sp2[i], sp[2 * i], sp[2 * i + 1]);
       }
-      TT_PH(2);
       tmem_st32u(s_addr, pk);                                  // P_t over the first 32 columns of S_t
       l = l * alpha + (((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7])));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&bars.p_full[t]));
-      TT_PH(3);
     };
     // tiles j < n_plain end at or before the first row's limit: every key of theirs is visible to every row
     const int n_plain = min(my_tiles, max(0, (t_min_limit[t] - kv_begin) / kTileKeys));
@@ -514,14 +472,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
     // ---- epilogue: O / l and LSE ----
     const float kLn2 = 0.6931471805599453f;
     if (my_tiles > 0) {
-      TT_BEGIN;
-      mbar_wait(smem_u32(&bars.o_full[t]), 0, abort_flag, P.status);
-      TT_END(tt_wait2);
+      mbar_wait(smem_u32(&bars.o_full[t]), 0, abort_flag, P.status, P.wait_limit_ns);
       tc_fence_after();
     }
-#ifdef TIDE_UMMA_TIMING
-    if (lane == 0 && (warp & 3) == 0) { TT_FLUSH(0, 1, 5); TT_PH_FLUSH(6); }   // counters 6..9: load, max, exp, store
-#endif
     const float inv = l > 0.f ? 1.f / l : 0.f;
     const float e2 = l > 0.f ? m + log2f(l) : -INFINITY;
     const long long orow = (long long)(seg.q_off + qi) * g.Hq + hd;

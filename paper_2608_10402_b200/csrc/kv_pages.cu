@@ -93,7 +93,7 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
   const int tokens = p.dyn ? p.grid_cap_tokens : p.n_tokens;
   if (tokens <= 0) return cudaSuccess;
   long long blocks = ((long long)tokens + kAppendThreads / 32 - 1) / (kAppendThreads / 32);
-  const long long cap = 148LL * 8 * 8;   // 8 resident blocks per SM, a few tokens per warp beyond this
+  const long long cap = (long long)sm_count() * 8 * 8;   // 8 resident blocks per SM, a few tokens per warp beyond this
   if (blocks > cap) blocks = cap;
   append_scatter_kernel<<<(unsigned)blocks, kAppendThreads, 0, s>>>(p);
   return cudaGetLastError();
@@ -146,7 +146,8 @@ cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int pos0,
   if (len <= 0) return cudaSuccess;
   const long long total = (long long)len * 2 * g.Hkv * (g.D / 8);
   long long blocks = (total + 255) / 256;
-  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  const long long cap = (long long)sm_count() * 64;
+  if (blocks > cap) blocks = cap;
   read_gather_kernel<<<(unsigned)blocks, 256, 0, s>>>(pool, table_row, pos0, len, out_k, out_v, g);
   return cudaGetLastError();
 }

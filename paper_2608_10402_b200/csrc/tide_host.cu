@@ -6,6 +6,7 @@
 // pops one page each time a token lands on slot 0 of a new logical page; release and truncate push pages
 // back last-to-first.  Every call validates completely before it changes anything.
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -21,8 +22,6 @@ namespace {
 constexpr int kSlots = 8;                    // staging ring depth
 constexpr size_t kSlotPageIds = 64 * 1024;   // most new page ids per upload
 constexpr int kSlotRecs = 2048;              // most append records per upload
-constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
-constexpr int kNumSms = 148;
 constexpr long long kPartRowsBase = 256 * 1024;
 constexpr long long kMinSavedBytesDefault = 64ll << 20;   // reads a batch must save before rows are planned as sharing groups
 constexpr int kStepSegStride = 2;   // each segment array of the step area holds up to 2 x max_batch_rows entries (rows + shared ranges)
@@ -104,6 +103,9 @@ struct tide_kv {
   int umma_min_rows = kDecodeTileRows + 1;  // packed rows from which a resume row takes the tcgen05 path (measured:
                                             // it beats the warp-MMA tile path from the first row beyond a decode item)
   int items_per_sm = kTargetItemsPerSm;  // work items the planner aims for per SM
+  int num_sms = 0;                       // multiprocessors of the handle's device
+  long long wait_limit_ns = kWaitLimitNsDefault;   // bound of every wait inside a kernel
+  bool drop_first_stage_once = false;    // test hook: armed by tide_tune, consumed by the next attention launch set
   // multi-layer step held between tide_step_begin and the tide_step_layer calls
   uint8_t* h_step = nullptr;   // pinned staging of the step area
   cudaEvent_t ev_step = nullptr;
@@ -288,6 +290,8 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->d_part_o = (float*)(kv->ws + lay.off_part_o);
   kv->d_part_lse = (float*)(kv->ws + lay.off_part_lse);
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
+  kv->num_sms = sm_count();
+  ok = ok && kv->num_sms > 0;
   ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
@@ -313,11 +317,6 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->pages.resize((size_t)cfg->max_tasks);
   kv->mark.assign((size_t)cfg->max_tasks, 0);
   kv->refcnt.assign((size_t)cfg->num_pages, 0);
-  if (const char* e = getenv("TIDE_ITEMS_PER_SM")) kv->items_per_sm = std::max(1, atoi(e));  // tuning knob
-  if (const char* e = getenv("TIDE_NO_GROUPING")) kv->no_grouping = atoi(e) != 0;   // planner switch for comparisons
-  if (const char* e = getenv("TIDE_MIN_SAVED_BYTES")) kv->min_saved_bytes = atoll(e);  // tuning knob
-  if (const char* e = getenv("TIDE_HOST_STEP_CHUNKS")) kv->host_step_chunks = std::max(0, atoi(e));  // tuning knob
-  if (const char* e = getenv("TIDE_UMMA_MIN_ROWS")) kv->umma_min_rows = std::max(17, atoi(e));  // tuning knob
   prime_free_stack(kv, cfg->free_order);
   *out = kv;
   return TIDE_OK;
@@ -854,7 +853,10 @@ static void find_share_groups(const tide_kv* kv, int32_t n_rows, const tide_row_
   for (int b = 0; b + 1 < n_rows; ++b) {
     if (rows[b].q_len != 1) continue;
     const auto& pg0 = kv->pages[rows[b].task];
-    int C = std::min<int>((int)pg0.size(), rows[b].ctx_len / g.S);
+    // Only pages that are full NOW can be shared: when a step is planned before its tokens are appended, a row's
+    // ctx_len counts the token that will land in the last page, and a shared partial page is replaced by a private
+    // copy before that token is written.
+    int C = std::min<int>((int)pg0.size(), std::min(rows[b].ctx_len, kv->len[rows[b].task]) / g.S);
     if (C < min_pages || kv->refcnt[(size_t)pg0[0]] < 2) continue;
     int m = 1;
     while (b + m < n_rows && m < max_m && rows[b + m].q_len == 1) {
@@ -863,7 +865,7 @@ static void find_share_groups(const tide_kv* kv, int32_t n_rows, const tide_row_
       for (int k = 0; k < m; ++k) repeat = repeat || rows[b + k].task == r.task;
       if (repeat) break;
       const auto& pg = kv->pages[r.task];
-      const int lim = std::min<int>(std::min<int>(C, (int)pg.size()), r.ctx_len / g.S);
+      const int lim = std::min<int>(std::min<int>(C, (int)pg.size()), std::min(r.ctx_len, kv->len[r.task]) / g.S);
       int lcp = 0;
       while (lcp < lim && pg[(size_t)lcp] == pg0[(size_t)lcp]) ++lcp;
       if (lcp < min_pages) break;
@@ -926,7 +928,7 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
   // decode rows are, whichever kernel its packed rows call for.
   auto shared_kind = [&](int R) { return kind_of(R); };
   for (const ShareGroup& sg : groups) w_dec += (long long)g.Hkv * sg.pages * g.S;
-  const long long target = (long long)kNumSms * kv->items_per_sm;
+  const long long target = (long long)kv->num_sms * kv->items_per_sm;
   long long chunk_dec = std::max<long long>(256, align_up((size_t)(w_dec / target + 1), kStageKeys));
   long long chunk_tile = (items_tile_nosplit >= target / 2)
                              ? (1LL << 30)
@@ -1073,6 +1075,9 @@ static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32
   ap.scale_log2e = scale * 1.4426950408889634f;
   ap.status = kv->d_status;
   ap.g = kv->g;
+  ap.wait_limit_ns = kv->wait_limit_ns;
+  ap.debug_drop_first_stage = kv->drop_first_stage_once ? 1 : 0;
+  kv->drop_first_stage_once = false;
   int64_t launches = 0;
   // dyn != nullptr: fixed launch shapes; the counts of the batch are read on the device (header of the step area)
   if (events) cudaEventRecord(kv->ev_attend[0], st);
@@ -1409,17 +1414,51 @@ int tide_phase_ms(tide_kv_t* kv, float* append_ms, float* decode_ms, float* tile
   return TIDE_OK;
 }
 
-// Read-only view of a handle for attend_static.cu (not part of the public header).
-int tide_internal_view(tide_kv_t* kv, Geom* g, const uint8_t** pool, const int32_t** table, int** status,
-                       const int32_t** len, const uint8_t** live, int32_t* max_tasks) {
+int tide_tune(tide_kv_t* kv, int knob, int64_t value) {
   if (kv == nullptr) return TIDE_ERR_INVALID_ARG;
-  *g = kv->g;
-  *pool = kv->pool;
-  *table = kv->d_table;
-  *status = kv->d_status;
-  *len = kv->len.data();
-  *live = kv->live.data();
-  *max_tasks = kv->cfg.max_tasks;
+  switch (knob) {
+    case TIDE_TUNE_ITEMS_PER_SM:
+      if (value < 1 || value > 64) return TIDE_ERR_INVALID_ARG;
+      kv->items_per_sm = (int)value;
+      break;
+    case TIDE_TUNE_GROUPING: kv->no_grouping = value == 0; break;
+    case TIDE_TUNE_MIN_SAVED_BYTES:
+      if (value < 0) return TIDE_ERR_INVALID_ARG;
+      kv->min_saved_bytes = value;
+      break;
+    case TIDE_TUNE_HOST_STEP_CHUNKS:
+      if (value < 0 || value > kMaxHostChunks) return TIDE_ERR_INVALID_ARG;
+      kv->host_step_chunks = (int)value;
+      break;
+    case TIDE_TUNE_UMMA_MIN_ROWS:
+      if (value <= kDecodeTileRows || value > 0x7fffffff) return TIDE_ERR_INVALID_ARG;
+      kv->umma_min_rows = (int)value;
+      break;
+    case TIDE_TUNE_WAIT_LIMIT_US:
+      if (value < 1 || value > 60ll * 1000 * 1000) return TIDE_ERR_INVALID_ARG;
+      kv->wait_limit_ns = value * 1000;
+      break;
+    case TIDE_TUNE_DROP_FIRST_STAGE: kv->drop_first_stage_once = value != 0; break;
+    default: return TIDE_ERR_INVALID_ARG;
+  }
+  kv->step_valid = false;   // a held plan was made with the old settings
+  return TIDE_OK;
+}
+
+// Read-only view of a handle for attend_static.cu (not part of the public header).
+int tide_internal_view(tide_kv_t* kv, tide::StaticView* v) {
+  if (kv == nullptr || v == nullptr) return TIDE_ERR_INVALID_ARG;
+  v->g = kv->g;
+  v->pool = kv->pool;
+  v->table = kv->d_table;
+  v->status = kv->d_status;
+  v->len = kv->len.data();
+  v->live = kv->live.data();
+  v->max_tasks = kv->cfg.max_tasks;
+  v->device = kv->device;
+  v->num_sms = kv->num_sms;
+  v->items_per_sm = kv->items_per_sm;
+  v->wait_limit_ns = kv->wait_limit_ns;
   return TIDE_OK;
 }
 
@@ -1441,3 +1480,23 @@ int tide_last_plan(tide_kv_t* kv, int64_t* decode_items, int64_t* prefill_items,
 }
 
 }  // extern "C"
+
+namespace tide {
+
+// Multiprocessors of the current device; asked of the runtime once per device.
+int sm_count() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int c = cache[dev].load(std::memory_order_relaxed);
+    if (c > 0) return c;
+  }
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 0;
+  if (dev >= 0 && dev < kMaxDevices) cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
+}  // namespace tide

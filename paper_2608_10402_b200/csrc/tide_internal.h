@@ -20,7 +20,8 @@ constexpr int kMaxSplits = 128;      // most KV splits of one row
 constexpr int kDecodeTileRows = 16;  // packed (query, head) rows per decode-style work item
 constexpr int kMmaTileRows = 64;     // packed rows per work item of the warp-MMA tile path
 constexpr int kUmmaTileRows = 128;   // packed rows per work item of the tcgen05 path
-constexpr long long kWaitLimitNs = 2000000000LL;  // bound of every in-kernel wait
+constexpr long long kWaitLimitNsDefault = 2000000000LL;  // bound of every in-kernel wait unless the handle says otherwise
+constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat finer balance (per-item set-up dominates)
 
 struct Geom {
   int Hq, Hkv, D, S, G;
@@ -73,6 +74,10 @@ struct AttendParams {
   // kernel reads n_items = dyn[0] and n_segs = dyn[1] from device memory; CTAs beyond n_items leave at once.
   const int32_t* dyn = nullptr;
   int grid_cap = 0;
+  long long wait_limit_ns = kWaitLimitNsDefault;   // bound of every wait inside the kernel
+  // Test hook for the bounded waits (never set in normal use): in work item 0 the producer leaves out its part
+  // of the first stage, so the consumers' wait for that stage runs out and the time-out path executes.
+  int debug_drop_first_stage = 0;
 };
 
 struct MergeParams {
@@ -108,6 +113,19 @@ struct AppendParams {
   int grid_cap_tokens = 0;
 };
 
+// What tide_attend_decode_static needs of a handle (filled by tide_internal_view in tide_host.cu).
+struct StaticView {
+  Geom g;
+  const uint8_t* pool;
+  const int32_t* table;
+  int* status;
+  const int32_t* len;      // host: resident tokens per task
+  const uint8_t* live;     // host
+  int32_t max_tasks;
+  int device, num_sms, items_per_sm;
+  long long wait_limit_ns;
+};
+
 cudaError_t launch_table_update(int32_t* table, const int32_t* idx, const int32_t* val, int n, cudaStream_t s);
 cudaError_t launch_upload(void* dst, const void* src_mapped_host, size_t bytes, cudaStream_t s);   // bytes % 4 == 0
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s);
@@ -120,6 +138,7 @@ cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);
 cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s);
 cudaError_t attend_kernels_init();
 cudaError_t attend_umma_init();
+int sm_count();   // multiprocessors of the current device (looked up once per device)
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------------------
@@ -145,19 +164,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Non-blocking test (try_wait may suspend the thread for a while when the phase is still open; a loop that
-// polls several barriers must not).
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -171,7 +177,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  `abort_flag` lives in shared memory: once any thread of the CTA has given up, every
 // later wait returns at once so that the CTA still walks its normal control flow to the end.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit_ns) {
   if (mbar_try(bar, parity)) return true;
   if (*abort_flag) return false;
   const long long t0 = global_ns();
@@ -179,7 +186,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   while (!mbar_try(bar, parity)) {
     if ((++spins & 255) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(status, (int)TIDE_ERR_DEVICE_TIMEOUT);
         return false;

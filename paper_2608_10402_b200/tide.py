@@ -18,6 +18,9 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNKNOWN_TASK, ERR_TASK_EXISTS, ERR_DUPLICATE_TASK = -1, -2, -3, -4
 ERR_NO_PAGES, ERR_TABLE_FULL, ERR_CTX_RANGE, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = -5, -6, -7, -8, -9, -10
 STATIC_MAX_ROWS = 64
+# knobs of tide_tune (tide_tune_t)
+(TUNE_ITEMS_PER_SM, TUNE_GROUPING, TUNE_MIN_SAVED_BYTES, TUNE_HOST_STEP_CHUNKS, TUNE_UMMA_MIN_ROWS, TUNE_WAIT_LIMIT_US,
+ TUNE_DROP_FIRST_STAGE) = range(7)
 
 
 class TideError(RuntimeError):
@@ -48,6 +51,7 @@ EXPORTS = [
     "tide_kv_task_len", "tide_kv_page_table", "tide_kv_usage", "tide_kv_read", "tide_status", "tide_last_plan",
     "tide_set_profiling", "tide_phase_ms", "tide_attend_decode_static", "tide_kv_release_many", "tide_kv_prune", "tide_kv_fork", "tide_kv_page_refs",
     "tide_kv_extend", "tide_kv_write", "tide_step_begin", "tide_step_layer", "tide_step_fix_grids", "tide_last_sharing",
+    "tide_tune",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -257,6 +261,9 @@ class TideKV:
 
     def status(self, stream=None):
         return lib.tide_status(self.handle, _stream(stream))
+
+    def tune(self, knob, value):
+        _check(lib.tide_tune(self.handle, ctypes.c_int(knob), ctypes.c_int64(int(value))), "tide_tune")
 
     def set_profiling(self, enable):
         _check(lib.tide_set_profiling(self.handle, ctypes.c_int(1 if enable else 0)), "tide_set_profiling")

@@ -130,7 +130,7 @@ def test_random_ops_with_forks_match_the_oracle_bit_for_bit():
 
 
 @pytest.mark.parametrize("geom", [(28, 4, 128, 16), (8, 2, 64, 16), (16, 1, 128, 32), (4, 4, 64, 32)])
-def test_decode_rows_of_forked_groups_read_their_shared_pages_once(geom, monkeypatch):
+def test_decode_rows_of_forked_groups_read_their_shared_pages_once(geom):
     """Groups of trajectories forked from one prompt, then decoding: the planner must treat each group's shared
     pages as one multi-query range (tide_last_sharing), and every row's result must still be plain attention over
     its whole context.  Group sizes around what one work item holds, members with and without tokens of their
@@ -138,11 +138,11 @@ def test_decode_rows_of_forked_groups_read_their_shared_pages_once(geom, monkeyp
     import torch
     from paper_2608_10402_b200 import tide
     HQ, HKV, D, S = geom
-    monkeypatch.setenv("TIDE_MIN_SAVED_BYTES", "0")      # small test batches: no minimum saving per batch
     rng = np.random.default_rng(HQ + D + S)
     scale = 1.0 / math.sqrt(D)
     NT = 40
     kv = tide.TideKV(HQ, HKV, D, S, 2000, NT, 200, NT, 64)
+    kv.tune(tide.TUNE_MIN_SAVED_BYTES, 0)      # small test batches: no minimum saving per batch
     orc = PagedKVOracle(2000, S, HKV, D, NT, 200)
 
     def app(ts, cnt):
@@ -202,4 +202,51 @@ def test_decode_rows_of_forked_groups_read_their_shared_pages_once(geom, monkeyp
     assert kv.last_sharing()["groups"] == 0
     ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
     H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, f"own table {geom}")
+    kv.close()
+
+
+def test_step_planned_before_its_append_does_not_share_a_page_that_is_about_to_be_copied():
+    """Forked tasks rolled back to one token short of a page edge INSIDE their shared pages, then stepped by one
+    token through tide_step_begin: the step is planned before the tokens are appended, the append gives each such
+    task a private copy of that last page, so the page must not be planned as part of the group's shared range -
+    otherwise every member but the first would read the first member's new token instead of its own."""
+    import torch
+    from paper_2608_10402_b200 import tide
+    rng = np.random.default_rng(2024)
+    P = 200
+    order = rng.permutation(P).astype(np.int32)
+    kv = tide.TideKV(HQ, HKV, D, S, P, 8, 64, 8, 64, free_order=order)
+    kv.tune(tide.TUNE_MIN_SAVED_BYTES, 0)
+    orc = PagedKVOracle(P, S, HKV, D, 8, 64, free_order=order)
+    scale = 1.0 / math.sqrt(D)
+    L0 = 20 * S
+    pk_, pv_ = inputs.normal_bf16(rng, (L0, HKV, D)), inputs.normal_bf16(rng, (L0, HKV, D))
+    for o in (kv, orc):
+        o.alloc(0)
+    kv.append([0], [0, L0], H.to_dev(pk_, torch), H.to_dev(pv_, torch))
+    orc.append([0], [0, L0], pk_, pv_)
+    for c in (1, 2, 3):
+        kv.fork(0, c)
+        orc.fork(0, c)
+    for c in (1, 2):                                         # 18 pages kept, the last one a shared page with one free slot
+        kv.truncate(c, 18 * S - 1)
+        orc.truncate(c, 18 * S - 1)
+    tasks = [1, 2, 3, 0]
+    rows = [(t, 1, orc.task_len(t) + 1) for t in tasks]
+    nk, nv, q = (inputs.normal_bf16(rng, (4, HKV, D)), inputs.normal_bf16(rng, (4, HKV, D)), inputs.normal_bf16(rng, (4, HQ, D)))
+    # make the new tokens matter: each task's own new key is the one its query likes best
+    qf = inputs.bf16_bits_to_f32(q)
+    for i in range(4):
+        for g in range(HKV):
+            nk[i, g] = inputs.f32_to_bf16_bits(qf[i, g * (HQ // HKV)] * 0.5)
+    out = torch.zeros((4, HQ, D), dtype=torch.int16, device="cuda")
+    lse = torch.zeros((4, HQ), dtype=torch.float32, device="cuda")
+    kv.step_begin(rows)
+    kv.step_layer(0, H.to_dev(nk, torch), H.to_dev(nv, torch), H.to_dev(q, torch), scale, out, lse)
+    assert kv.status() == tide.OK
+    assert kv.last_sharing()["groups"] >= 1, "the case is meant to be planned as a sharing group"
+    orc.append(tasks, np.arange(5), nk, nv)
+    _same(kv, orc, tasks)
+    ref_o, ref_l = cbuild.attend_paged(orc, rows, q, scale)
+    H.check_outputs(H.from_dev(out), lse.cpu().numpy(), ref_o, ref_l, "step over a rolled-back group")
     kv.close()

@@ -1,4 +1,4 @@
-"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times (same library calls:
+"""GPU parity at the workloads' full sizes, in the launch configuration bench.py times (same library calls:
 per-task prefix appends, one step append, one tide_attend).  Page tables, lengths and cache bits of every task
 are compared exactly; attention outputs are compared on a stratified sample of (row, query) items the float64
 oracle computes one by one (every decode row; first / last / page-boundary / image-text-boundary and random

@@ -106,6 +106,8 @@ def _run_steps(seed, n_ops, tide, torch):
     P, NT, MAXP = 400, 8, 60
     order = rng.permutation(P).astype(np.int32)
     kv = tide.TideKV(HQ, HKV, D, S, P, NT, MAXP, 2 * NT, 4096, free_order=order, num_layers=L)
+    # odd seeds: no minimum saving per batch, so that forked rows are planned as sharing groups whenever they can be
+    kv.tune(tide.TUNE_MIN_SAVED_BYTES, 0 if seed % 2 else 64 << 20)
     orc = LayeredKVOracle(L, num_pages=P, page_size=S, num_kv_heads=HKV, head_dim=D, max_tasks=NT, max_pages_per_task=MAXP, free_order=order)
     scale = 1 / math.sqrt(D)
     n_att = 0
@@ -166,7 +168,7 @@ def _run_steps(seed, n_ops, tide, torch):
     return n_att
 
 
-def test_random_steps_and_windows_match_the_oracle(monkeypatch):
+def test_random_steps_and_windows_match_the_oracle():
     """Random geometries (head counts, head size, page size, layers); steps through tide_step_begin /
     tide_step_layer with decode and resume rows, attention over arbitrary windows of live tasks, interleaved with
     forks, truncates, prunes and releases; every attention result against the float64 oracle."""
@@ -174,7 +176,5 @@ def test_random_steps_and_windows_match_the_oracle(monkeypatch):
     from paper_2608_10402_b200 import tide
     checks = 0
     for seed in range(8):
-        # odd seeds: no minimum saving per batch, so that forked rows are planned as sharing groups whenever they can be
-        monkeypatch.setenv("TIDE_MIN_SAVED_BYTES", "0" if seed % 2 else str(64 << 20))
         checks += _run_steps(seed, 80, tide, torch)
     assert checks > 100

@@ -135,11 +135,14 @@ def test_ctb_invariant_on_gpu_resume_equals_recompute(env):
         o_res = torch.zeros((n, w.Hq, w.D), dtype=torch.int16, device="cuda")
         l_res = torch.zeros((n, w.Hq), dtype=torch.float32, device="cuda")
         kv.attend([(t, n, L)], H.to_dev(qf[L - n:], torch), w.scale, o_res, l_res)
+        # both passes against the oracle's from-scratch pass first: the resumed rows must equal ITS last n rows
+        ref_o, ref_l = H.cbuild.attend_paged(c, [(t, L, L)], qf, w.scale)
+        H.check_outputs(H.from_dev(o_all), l_all.cpu().numpy(), ref_o, ref_l, "from-scratch pass")
+        H.check_outputs(H.from_dev(o_res), l_res.cpu().numpy(), ref_o[L - n:], ref_l[L - n:], "resumed chunk vs from-scratch oracle")
+        # and, as a second check, against each other
         a = H.oa.bf16_bits_to_f64(H.from_dev(o_all))[L - n:]
         r = H.oa.bf16_bits_to_f64(H.from_dev(o_res))
         assert np.abs(a - r).max() <= 2e-2 and np.abs(l_all.cpu().numpy()[L - n:] - l_res.cpu().numpy()).max() < 1e-3
-        ref_o, ref_l = H.cbuild.attend_paged(c, [(t, L, L)], qf, w.scale)
-        H.check_outputs(H.from_dev(o_all), l_all.cpu().numpy(), ref_o, ref_l, "from-scratch pass")
     assert kv.status() == tide.OK
     kv.close()
 
@@ -211,11 +214,10 @@ def test_append_leaves_neighbouring_slots_untouched(env):
 
 
 @pytest.mark.parametrize("groups", [0, 3, 8])
-def test_step_host_matches_append_then_attend(env, groups, monkeypatch):
+def test_step_host_matches_append_then_attend(env, groups):
     # groups > 0 forces the step to be cut into that many row groups whose copies and kernels overlap (what large
     # steps do by themselves); pages, cache bits and outputs must not depend on the cut
     tide, torch = env
-    monkeypatch.setenv("TIDE_HOST_STEP_CHUNKS", str(groups))
     w = inputs.make_workload(1)
     kv_bits = [w.task_kv(b) for b in range(w.B)]
     q_bits = np.concatenate([w.task_q(b) for b in range(w.B)])
@@ -223,6 +225,7 @@ def test_step_host_matches_append_then_attend(env, groups, monkeypatch):
     total_q = int(w.n_new.sum())
     kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task, w.B, total_q,
                      free_order=w.free_order)
+    kv.tune(tide.TUNE_HOST_STEP_CHUNKS, groups)
     for b in range(w.B):
         kv.alloc(int(w.task[b]))
     for b in range(w.B):

@@ -2,9 +2,9 @@
 global-mode CUDA graph capture, processes whose allocator already owns the device, steps that must avoid
 cudaMalloc's device-wide synchronisation).  Its split-KV scratch is a fixed array inside the library.
 
-Checked here through the C ABI against tide_attend on the same cache and queries, on two calls in a row
-(the second call reuses the array with the first call's leftovers in it), within the tolerance the parity
-tests use.  Collected last on purpose: a run that stops at the first failure has then run everything else.
+Checked here through the C ABI against the float64 oracle and against tide_attend on the same cache and
+queries, on two calls in a row (the second call reuses the array with the first call's leftovers in it), within
+the tolerance the parity tests use.  Collected last on purpose: a run that stops at the first failure has then run everything else.
 """
 import numpy as np
 import pytest
@@ -37,6 +37,9 @@ def test_static_scratch_attend_matches_tide_attend_twice():
         got_l = torch.zeros_like(ref_l)
         kv.attend_decode_static(rows, q, w.scale, got_o, got_l)
         assert kv.status() == tide.OK
+        q_bits = H.from_dev(q)
+        want_o, want_l = H.oracle_attend(c, w, q_bits)
+        H.check_outputs(H.from_dev(got_o), got_l.cpu().numpy(), want_o, want_l, f"static entry point, call {call}")
         a = H.oa.bf16_bits_to_f64(H.from_dev(got_o))
         b = H.oa.bf16_bits_to_f64(H.from_dev(ref_o))
         assert np.isfinite(a).all()
