@@ -29,10 +29,6 @@ struct MmaCfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
 };
 
-__device__ __forceinline__ int blk_chunk_offset(int S, int slot, int c) {
-  return (c >> 3) * (S * 128) + slot * 128 + (((c & 7) ^ (slot & 7)) << 4);
-}
-
 template <int D, bool DECODE>
 __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const AttendParams P) {
   constexpr int KS = D / 16;                 // k-steps of Q.K^T
@@ -201,7 +197,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
 #pragma unroll
             for (int k2 = 0; k2 < KS / 2; ++k2) {
               uint32_t b0, b1, b2, b3;
-              ldsm_x4(pbase + blk_chunk_offset(g.S, slot_row, k2 * 4 + (lane >> 3)), b0, b1, b2, b3);
+              ldsm_x4(pbase + blk_offset(g, slot_row, 0, k2 * 4 + (lane >> 3)), b0, b1, b2, b3);
               mma_bf16(acc, qa[2 * k2], b0, b1);
               mma_bf16(acc, qa[2 * k2 + 1], b2, b3);
             }
@@ -257,7 +253,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
       for (int b = 0; b < STEP_KB; ++b) {
         if (b < nkb) {
           const int koff = (kb_first + b) * 16;
-          const uint32_t vbase = stage + (koff / g.S) * g.head_bytes + g.kblock_bytes;
+          const uint32_t vbase = stage + (koff / g.S) * g.head_bytes;   // the page block; V parts through blk_offset(.., 1, ..)
           const int row0 = koff % g.S;
           const int blk_key0 = key0 + koff;
           if (blk_key0 + 16 > kv_end) {
@@ -267,7 +263,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
             uint8_t* vgen = smem_gen + (vbase - smem_base);
             for (int idx = lane; idx < (16 - first) * (D / 8); idx += 32) {
               const int rr = row0 + first + idx / (D / 8), c = idx % (D / 8);
-              *reinterpret_cast<uint4*>(vgen + blk_chunk_offset(g.S, rr, c)) = make_uint4(0, 0, 0, 0);
+              *reinterpret_cast<uint4*>(vgen + blk_offset(g, rr, 1, c)) = make_uint4(0, 0, 0, 0);
             }
             __syncwarp();
           }
@@ -280,7 +276,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
 #pragma unroll
           for (int n2 = 0; n2 < NT / 2; ++n2) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4_t(vbase + blk_chunk_offset(g.S, vrow, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
+            ldsm_x4_t(vbase + blk_offset(g, vrow, 1, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
             mma_bf16(o[2 * n2], pa, b0, b1);
             mma_bf16(o[2 * n2 + 1], pa, b2, b3);
           }

@@ -9,9 +9,11 @@
 // This is a dense contraction (n*G x ctx x D), so it is bound by the tensor pipe: 4*D flops per visible
 // (packed row, key) pair against Hkv*D*4 bytes per key shared by all packed rows.
 //
-// CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warps 8, 10 and 11
-// stream K and V tiles of 64 keys (page blocks arrive pre-swizzled, so plain 1-D bulk copies build the canonical
-// 128-byte-swizzled operand tiles); one lane of warp 9 issues every MMA.  TMEM (512 columns):
+// CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warp 8 streams tiles of
+// 64 keys, one plain 1-D bulk copy per (page, head) block (blocks are stored as the canonical 128-byte-swizzled
+// core-matrix atoms, K and V of 8 keys side by side, so the blocks of a tile laid one after the other ARE the K-major
+// K operand and the MN-major V operand, a uniform 4 KB between 8-key groups); one lane of warp 9 issues every MMA.
+// TMEM (512 columns):
 //   Q_A Q_B   2 x 64   the queries as packed bf16, staged once per item
 //   S_A S_B   2 x 64   fp32 logits of one 64-key tile; P (packed bf16) overwrites the first 32 columns
 //   O_A O_B   2 x 128  fp32 output accumulators
@@ -34,12 +36,11 @@ namespace umma {
 
 constexpr int D = 128;
 constexpr int kTileKeys = 64;
-constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {three producer warps and the MMA issuer}
+constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer warp 8, MMA issuer warp 9, two idle warps}
 constexpr int kNumBuf = 6;                          // ring of (K tile, V tile) slots
-constexpr int kProducerWarps = 3;                   // warps 8, 10, 11
-constexpr int kTileBytes = kTileKeys * D * 2;       // one K or V tile: 16 KB
-constexpr int kSlotBytes = 2 * kTileBytes;          // K tile then V tile
-constexpr int kSlabBytes = kTileKeys * 128;         // 64 rows x 128 bytes
+constexpr int kKvBytes = (D / 64) * 1024;           // K (or V) of one 8-key group: two 1-KB atoms
+constexpr int kGroupBytes = 2 * kKvBytes;           // one 8-key group: K then V
+constexpr int kSlotBytes = (kTileKeys / 8) * kGroupBytes;   // one 64-key tile, K and V: 32 KB
 constexpr int kSmemBytes = kNumBuf * kSlotBytes + 1024;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
 constexpr uint32_t kColQ = 0, kColS = 128, kColO = 256;
@@ -206,7 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), kProducerWarps); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
+    for (int i = 0; i < kNumBuf; ++i) { mbar_init(smem_u32(&bars.kv_full[i]), 1); mbar_init(smem_u32(&bars.kv_empty[i]), 1); }
     mbar_init(smem_u32(&bars.q_full), 256);
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
@@ -231,16 +232,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   // more than that: 256 x 224 + 128 x 56 = 384 x 168.  (An over-subscribed .inc waits for ever.)
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    if (warp != 9) {
-      // ================= producers: K0 V0 K1 V1 ... into the ring =================
-      // Three warps (8, 10, 11) share the copies of every tile: a bulk copy costs its warp about 55 cycles of
-      // issue whatever its size, so the 16 copies of a tile from one warp (~1400 cycles per 32 KB measured) were
-      // most of a tile pair's time; each warp announces its own bytes on the slot's barrier.
-      const int pw = warp == 8 ? 0 : warp - 9;                 // 0, 1, 2
+    if (warp == 8) {
+      // ================= producer: one copy per (page, head) block into the ring =================
       if (n_tiles > 0) {
         const int pages_per_tile = kTileKeys / g.S;
-        const int slab_block = g.S * 128;                    // bytes of one slab of a page block
-        const int copies = pages_per_tile * 2;               // (page, slab) pairs per operand tile
         // page ids are fetched 32 logical pages at a time, one per lane, a whole group ahead of their use,
         // so that no bulk copy waits for a dependent page-table load
         const int tiles_per_group = 32 / pages_per_tile;
@@ -251,7 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           return lp < g.max_pages_per_task ? trow[lp] : 0;
         };
         int ids_cur = load_ids(0), ids_nxt = load_ids(1), cur_grp = 0;
-        int issued = 0;                                        // tiles this warp has issued its copies of
+        int issued = 0;                                        // tiles whose copies were issued
         for (int j = 0; j < n_tiles; ++j) {
           const int buf = j % kNumBuf, use = j / kNumBuf;
           const int grp = j / tiles_per_group;
@@ -259,28 +254,21 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           // a wait that gave up means the ring can no longer be trusted: issue nothing more
           if (use > 0 && !mbar_wait(smem_u32(&bars.kv_empty[buf]), (use - 1) & 1, abort_flag, P.status, P.wait_limit_ns)) break;
           issued = j + 1;
-          if (P.debug_drop_first_stage != 0 && item == 0 && j == 0 && pw == 0) continue;   // test hook: this warp's part of tile 0 never arrives
+          if (P.debug_drop_first_stage != 0 && item == 0 && j == 0) continue;   // test hook: tile 0 never arrives
           const int key0 = kv_begin + j * kTileKeys;
           const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
           const uint32_t bar = smem_u32(&bars.kv_full[buf]);
-          // lanes [0, copies) fetch the K pieces, lanes [copies, 2*copies) the V pieces of this tile; every third one here
-          const int is_v = lane >= copies ? 1 : 0;
-          const int c = lane - is_v * copies;
-          const int pg = c >> 1, slab = c & 1;
-          const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + pg) & 31);
-          const bool mine = lane < 2 * copies && pg < npages && lane % kProducerWarps == pw;
-          const uint32_t n_mine = (uint32_t)__popc(__ballot_sync(0xffffffffu, mine));
-          if (lane == 0) mbar_expect_tx(bar, n_mine * (uint32_t)slab_block);
-          if (mine) {
-            const uint8_t* src = P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes + is_v * g.kblock_bytes + slab * slab_block;
-            bulk_g2s(smem_base + buf * kSlotBytes + is_v * kTileBytes + slab * kSlabBytes + pg * slab_block, src, (uint32_t)slab_block, bar);
-          }
+          const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + lane) & 31);
+          if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * g.head_bytes));
+          __syncwarp();
+          if (lane < npages)
+            bulk_g2s(smem_base + buf * kSlotBytes + lane * g.head_bytes, P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes,
+                     (uint32_t)g.head_bytes, bar);
         }
         if (*abort_flag && lane == 0) {
-          // a wait gave up somewhere: this warp does not leave while copies it issued into the CTA's shared memory
-          // can still be landing.  Those are among its last kNumBuf tiles (an older one was consumed before its slot
-          // was refilled); a tile's barrier completes when all three producer warps' parts are in, and each wait is
-          // bounded like every other (a tile another warp never issued its part of runs into that bound).
+          // a wait gave up somewhere: do not leave while copies into this CTA's shared memory can still be landing.
+          // Those are among the last kNumBuf tiles issued (an older one was consumed before its slot was refilled);
+          // each wait is bounded like every other.
           for (int idx = max(0, issued - kNumBuf); idx < issued; ++idx) {
             const uint32_t bar = smem_u32(&bars.kv_full[idx % kNumBuf]);
             const long long t0 = global_ns();
@@ -298,14 +286,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
             mma_ts(tmem + kColS + t * 64, tmem + kColQ + t * 64 + ks * 8,
-                   make_desc(kbuf + (ks >> 2) * kSlabBytes + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+                   make_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, kGroupBytes), kIdescQK, ks > 0);
           mma_commit(smem_u32(&bars.s_full[t]));
         };
         auto issue_pv = [&](int t, int j) {
-          const uint32_t vbuf = smem_base + (j % kNumBuf) * kSlotBytes + kTileBytes;
+          const uint32_t vbuf = smem_base + (j % kNumBuf) * kSlotBytes + kKvBytes;
 #pragma unroll
           for (int ks = 0; ks < kTileKeys / 16; ++ks)
-            mma_ts(tmem + kColO + t * 128, tmem + kColS + t * 64 + ks * 8, make_desc(vbuf + ks * 2048, kSlabBytes, 1024), kIdescPV,
+            mma_ts(tmem + kColO + t * 128, tmem + kColS + t * 64 + ks * 8, make_desc(vbuf + ks * 2 * kGroupBytes, 1024, kGroupBytes), kIdescPV,
                    (j > 0 || ks > 0) ? 1u : 0u);
         };
         auto wait_full = [&](int idx) {
@@ -319,10 +307,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
             // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
             // them so that weight 0 times leftover bits cannot produce NaN
             const int first = kv_end - (kv_begin + j * kTileKeys);
-            uint8_t* vgen = smem_gen + (j % kNumBuf) * kSlotBytes + kTileBytes;
+            uint8_t* vgen = smem_gen + (j % kNumBuf) * kSlotBytes + kKvBytes;
             for (int i = lane; i < (kTileKeys - first) * 16; i += 32) {
-              const int rr = first + (i >> 4), c = i & 15;
-              *reinterpret_cast<uint4*>(vgen + (c >> 3) * kSlabBytes + rr * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+              const int rr = first + (i >> 4), c = i & 15;     // whole rows are cleared, so the swizzle does not matter
+              *reinterpret_cast<uint4*>(vgen + (rr >> 3) * kGroupBytes + (c >> 3) * 1024 + (rr & 7) * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
             }
             fence_async_smem();
             __syncwarp();

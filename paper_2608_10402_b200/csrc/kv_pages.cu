@@ -37,65 +37,113 @@ cudaError_t launch_upload(void* dst, const void* src_mapped_host, size_t bytes, 
   return cudaGetLastError();
 }
 
-// Byte offset of 16-byte chunk `c` (c = d / 8) of slot `slot` inside a K or V block.
-__device__ __forceinline__ int chunk_offset(int S, int slot, int c) {
-  return (c >> 3) * (S * 128) + slot * 128 + (((c & 7) ^ (slot & 7)) << 4);
-}
-
 constexpr int kAppendThreads = 256;
+constexpr int kAppendWarps = kAppendThreads / 32;
 constexpr int kAppendMaxRecsSmem = 1024;
+constexpr int kAppendLoadsInFlight = 8;    // 16-byte loads a lane has in flight before its first store
 
-// One warp per token at a time: the record lookup, the page-table read and the slot arithmetic happen once per
-// token (warp-uniform), then the lanes copy the token's 16-byte chunks, ordered [K|V][kv_head][chunk], so a warp
-// reads 512 contiguous source bytes and writes four full 128-byte lines per pass.  D/8 is a power of two, so the
-// per-chunk index split needs no division.
-__global__ void __launch_bounds__(kAppendThreads) append_scatter_kernel(const AppendParams P) {
+// One warp per token at a time: the record lookup, the page lookup and the slot arithmetic happen once per token
+// (warp-uniform), then the lanes copy the token's 16-byte chunks, ordered [K|V][kv_head][chunk]: a warp reads 512
+// contiguous source bytes and writes four full 128-byte lines per pass.  A copy like this is bound by how many
+// bytes are in flight, so a warp takes several tokens per round and issues all their loads (eight per lane)
+// before the first store.  CPL = chunks per lane per token when a token is a multiple of 32 chunks (0: any
+// count, plain loop).  The same launch first applies the page-table delta of the append, if it is given one; the
+// pages that delta brings are then taken from the delta itself, not from the table (no ordering between thread
+// blocks is needed).
+template <int CPL>
+__global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_kernel(const AppendParams P) {
   __shared__ int32_t s_tok0[kAppendMaxRecsSmem];
   const int n_recs = P.dyn ? P.dyn[0] : P.n_recs;
   const int n_tokens = P.dyn ? P.dyn[1] : P.n_tokens;
+  for (int i = blockIdx.x * kAppendThreads + threadIdx.x; i < P.n_upd; i += gridDim.x * kAppendThreads)
+    P.table_rw[P.upd_idx[i]] = P.upd_val[i];
   const bool in_smem = n_recs <= kAppendMaxRecsSmem;
   if (in_smem) {
     for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = P.recs[i].tok0;
     __syncthreads();
   }
+  const Geom& g = P.g;
   const int lane = threadIdx.x & 31;
-  const int cpr = P.g.D >> 3;                 // chunks per (token, head) row: 8 or 16
+  const int cpr = g.D >> 3;                   // chunks per (token, head) row: 8 or 16
   const int shift = cpr == 16 ? 4 : 3;
-  const int rows2 = 2 * P.g.Hkv;              // K rows then V rows of one token
-  const int cpt = rows2 * cpr;                // chunks per token
-  const int warps_total = gridDim.x * (kAppendThreads / 32);
-  for (int tok = blockIdx.x * (kAppendThreads / 32) + (threadIdx.x >> 5); tok < n_tokens; tok += warps_total) {
+  const int cpt = 2 * g.Hkv * cpr;            // chunks per token: K rows then V rows
+  const int warps_total = gridDim.x * kAppendWarps;
+  const int warp_id = blockIdx.x * kAppendWarps + (threadIdx.x >> 5);
+
+  // where token `tok` goes: the base of its page (slot offsets are added per chunk) and its slot
+  auto locate = [&](int tok, int& slot) -> uint8_t* {
     int r;
     if (in_smem) r = find_segment(n_recs, tok, [&](int i) { return s_tok0[i]; });
     else r = find_segment(n_recs, tok, [&](int i) { return P.recs[i].tok0; });
     const AppendRec rec = P.recs[r];
     const int pos = rec.pos0 + (tok - rec.tok0);
-    const int lp = pos / P.g.S, slot = pos - lp * P.g.S;
-    const long long page = P.table[rec.table_off + lp];
-    uint8_t* page_base = P.pool + page * P.g.page_bytes + slot * 128;
-    const uint16_t* src_k = P.new_k + (long long)tok * P.g.Hkv * P.g.D;
-    const uint16_t* src_v = P.new_v + (long long)tok * P.g.Hkv * P.g.D;
-    const int sw = slot & 7;
-    for (int c = lane; c < cpt; c += 32) {
-      const int cc = c & (cpr - 1);
-      const int row = c >> shift;               // 0 .. 2*Hkv-1
-      const int kv = row >= P.g.Hkv ? 1 : 0;
-      const int h = row - kv * P.g.Hkv;
-      const uint16_t* src = (kv ? src_v : src_k) + h * P.g.D + cc * 8;
-      uint8_t* dst = page_base + (long long)h * P.g.head_bytes + kv * P.g.kblock_bytes + (cc >> 3) * (P.g.S * 128) +
-                     (((cc & 7) ^ sw) << 4);
-      *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    const int lp = pos / g.S;
+    slot = pos - lp * g.S;
+    const long long page = lp >= rec.new_lp0 ? P.upd_val[rec.new_off + (lp - rec.new_lp0)] : P.table[rec.table_off + lp];
+    return P.pool + page * g.page_bytes;
+  };
+  // chunk c of a token: source address and offset inside the page
+  auto src_of = [&](int tok, int c) -> const uint4* {
+    const int row = c >> shift, cc = c & (cpr - 1);
+    const int kv = row >= g.Hkv ? 1 : 0, h = row - kv * g.Hkv;
+    return reinterpret_cast<const uint4*>((kv ? P.new_v : P.new_k) + ((long long)tok * g.Hkv + h) * g.D + cc * 8);
+  };
+  auto dst_off = [&](int slot, int c) -> long long {
+    const int row = c >> shift, cc = c & (cpr - 1);
+    const int kv = row >= g.Hkv ? 1 : 0, h = row - kv * g.Hkv;
+    return (long long)h * g.head_bytes + blk_offset(g, slot, kv, cc);
+  };
+
+  if constexpr (CPL > 0) {
+    constexpr int TOK = kAppendLoadsInFlight / CPL;          // tokens per warp per round
+    for (int t0 = warp_id; t0 < n_tokens; t0 += warps_total * TOK) {
+      uint4 v[TOK][CPL];
+      uint8_t* base[TOK];
+      int slot[TOK];
+#pragma unroll
+      for (int u = 0; u < TOK; ++u) {
+        const int tok = t0 + u * warps_total;
+        base[u] = nullptr;
+        if (tok < n_tokens) {
+          base[u] = locate(tok, slot[u]);
+#pragma unroll
+          for (int i = 0; i < CPL; ++i) v[u][i] = __ldg(src_of(tok, lane + 32 * i));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < TOK; ++u) {
+        if (base[u] != nullptr) {
+#pragma unroll
+          for (int i = 0; i < CPL; ++i) *reinterpret_cast<uint4*>(base[u] + dst_off(slot[u], lane + 32 * i)) = v[u][i];
+        }
+      }
+    }
+  } else {
+    for (int tok = warp_id; tok < n_tokens; tok += warps_total) {
+      int slot;
+      uint8_t* base = locate(tok, slot);
+      for (int c = lane; c < cpt; c += 32) *reinterpret_cast<uint4*>(base + dst_off(slot, c)) = __ldg(src_of(tok, c));
     }
   }
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
   const int tokens = p.dyn ? p.grid_cap_tokens : p.n_tokens;
-  if (tokens <= 0) return cudaSuccess;
-  long long blocks = ((long long)tokens + kAppendThreads / 32 - 1) / (kAppendThreads / 32);
-  const long long cap = (long long)sm_count() * 8 * 8;   // 8 resident blocks per SM, a few tokens per warp beyond this
-  if (blocks > cap) blocks = cap;
-  append_scatter_kernel<<<(unsigned)blocks, kAppendThreads, 0, s>>>(p);
+  if (tokens <= 0 && p.n_upd <= 0) return cudaSuccess;
+  const int cpt = 2 * p.g.Hkv * (p.g.D / 8);
+  const int cpl = cpt % 32 == 0 ? cpt / 32 : 0;
+  const int tok_per_round = (cpl == 1 || cpl == 2 || cpl == 4 || cpl == 8) ? kAppendLoadsInFlight / cpl : 1;
+  long long blocks = ((long long)std::max(tokens, 1) + kAppendWarps * tok_per_round - 1) / (kAppendWarps * tok_per_round);
+  const long long cap = (long long)sm_count() * 3;   // the resident blocks; each warp loops over rounds beyond this
+  blocks = std::max<long long>(1, std::min(blocks, cap));
+  const dim3 grid((unsigned)blocks);
+  switch (cpl) {
+    case 1: append_scatter_kernel<1><<<grid, kAppendThreads, 0, s>>>(p); break;
+    case 2: append_scatter_kernel<2><<<grid, kAppendThreads, 0, s>>>(p); break;
+    case 4: append_scatter_kernel<4><<<grid, kAppendThreads, 0, s>>>(p); break;
+    case 8: append_scatter_kernel<8><<<grid, kAppendThreads, 0, s>>>(p); break;
+    default: append_scatter_kernel<0><<<grid, kAppendThreads, 0, s>>>(p); break;
+  }
   return cudaGetLastError();
 }
 
@@ -134,8 +182,7 @@ __global__ void read_gather_kernel(const uint8_t* __restrict__ pool, const int32
     const int pos = pos0 + row;
     const int lp = pos / g.S, slot = pos - lp * g.S;
     const long long page = table_row[lp];
-    const uint8_t* src = pool + page * g.page_bytes + (long long)h * g.head_bytes + kv * g.kblock_bytes +
-                         chunk_offset(g.S, slot, c);
+    const uint8_t* src = pool + page * g.page_bytes + (long long)h * g.head_bytes + blk_offset(g, slot, kv, c);
     uint16_t* dst = (kv ? out_v : out_k) + ((long long)row * g.Hkv + h) * g.D + c * 8;
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }

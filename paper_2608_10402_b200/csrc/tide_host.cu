@@ -7,6 +7,7 @@
 // back last-to-first.  Every call validates completely before it changes anything.
 #include <algorithm>
 #include <atomic>
+#include <climits>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -55,6 +56,14 @@ struct PlanHost {
   size_t n_all() const { return seg_dec.size() + seg_tile.size() + seg_umma.size() + seg_merge.size(); }
 };
 
+// What an extension of tasks did, as host arrays that are reused from call to call.
+struct ExtendOut {
+  std::vector<int32_t> idx, val;           // page-table delta: table[idx[i]] = val[i]
+  std::vector<int32_t> cpy_src, cpy_dst;   // private copies of shared partial pages (old page -> new page)
+  std::vector<int32_t> new_lp0, new_off;   // per task of the call: first logical page the delta brings, its place in val
+  void clear() { idx.clear(); val.clear(); cpy_src.clear(); cpy_dst.clear(); new_lp0.clear(); new_off.clear(); }
+};
+
 struct Slot {
   uint8_t* host = nullptr;
   uint8_t* dev = nullptr;
@@ -86,6 +95,7 @@ struct tide_kv {
   std::vector<int32_t> len;
   std::vector<std::vector<int32_t>> pages;
   std::vector<int32_t> refcnt;  // per physical page: how many tasks hold it (0 = free)
+  ExtendOut ext;              // result of the most recent extension
   std::vector<int32_t> mark;  // scratch for duplicate detection
   int32_t mark_gen = 0;
   int64_t used_tokens = 0;
@@ -144,8 +154,9 @@ Geom make_geom(const tide_kv_config_t* c) {
   Geom g;
   g.Hq = c->num_q_heads; g.Hkv = c->num_kv_heads; g.D = c->head_dim; g.S = c->page_size; g.G = g.Hq / g.Hkv;
   g.max_pages_per_task = c->max_pages_per_task;
-  g.kblock_bytes = g.D * g.S * 2;
-  g.head_bytes = 2 * g.kblock_bytes;
+  g.kv_bytes = (g.D / 64) * 1024;
+  g.group_bytes = 2 * g.kv_bytes;
+  g.head_bytes = (g.S / 8) * g.group_bytes;
   g.page_bytes = (long long)g.head_bytes * g.Hkv;
   return g;
 }
@@ -455,99 +466,108 @@ static int check_extend(const tide_kv* kv, int32_t n_tasks, const int32_t* task_
   return need > (long long)kv->free_stack.size() ? TIDE_ERR_NO_PAGES : TIDE_OK;
 }
 
-// Grows task_ids[j] by indptr[j+1]-indptr[j] tokens: host tables first, then the device page table, in uploads of
-// bounded size.  No K/V is written.  A task that ends inside a page that other tasks hold gets a private copy of
-// that page before its other pages are taken: with cow_out == nullptr the copy runs here on every layer, otherwise
-// the (old, new) page pairs are handed back and the caller copies (it may have to read the old pages first).
+// Grows task_ids[j] by indptr[j+1]-indptr[j] tokens in the host tables and records, in kv->ext, what the device
+// still has to be told: the page-table delta and the private copies of shared partial pages (a task that ends inside
+// a page that other tasks hold gets a private copy of that page before its other pages are taken).  No device work.
 // The task list must have passed check_task_list.
-static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, cudaStream_t st,
-                        std::vector<int32_t>* cow_out) {
+static int extend_bookkeeping(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr) {
   const Geom& g = kv->g;
-  int rc = check_extend(kv, n_tasks, task_ids, indptr);
+  const int rc = check_extend(kv, n_tasks, task_ids, indptr);
   if (rc != TIDE_OK) return rc;
-
   // ---- mutation ----
   kv->step_valid = false;
-  Slot* slot = nullptr;
-  int32_t *idx = nullptr, *val = nullptr, *cpy_src = nullptr, *cpy_dst = nullptr;
-  size_t n_ids = 0;
-  int n_cpy = 0;
-  auto open_slot = [&]() -> int {
-    if (slot != nullptr) return TIDE_OK;
-    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
-    idx = (int32_t*)(slot->host + 256 + (size_t)kSlotRecs * sizeof(AppendRec));
-    val = idx + kSlotPageIds;
-    cpy_src = val + kSlotPageIds;
-    cpy_dst = cpy_src + kSlotRecs;
-    return TIDE_OK;
-  };
-  auto flush = [&]() -> int {
-    if (slot == nullptr) return TIDE_OK;
-    if (n_ids > 0) {
-      uint8_t* didx = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec);
-      if (upload(kv, didx, idx, n_ids * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (upload(kv, didx + kSlotPageIds * 4, val, n_ids * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (launch_table_update(kv->d_table, (const int32_t*)didx, (const int32_t*)(didx + kSlotPageIds * 4), (int)n_ids, st) != cudaSuccess)
-        return TIDE_ERR_CUDA;
-      ++kv->append_launches;
-    }
-    if (n_cpy > 0 && cow_out == nullptr) {
-      uint8_t* dcpy = slot->dev + 256 + (size_t)kSlotRecs * sizeof(AppendRec) + kSlotPageIds * 8;
-      if (upload(kv, dcpy, cpy_src, (size_t)n_cpy * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      if (upload(kv, dcpy + (size_t)kSlotRecs * 4, cpy_dst, (size_t)n_cpy * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
-      for (int l = 0; l < kv->cfg.num_layers; ++l) {
-        if (launch_copy_pages(kv->layer_pool(l), (const int32_t*)dcpy, (const int32_t*)(dcpy + (size_t)kSlotRecs * 4), n_cpy,
-                              g.page_bytes, st) != cudaSuccess)
-          return TIDE_ERR_CUDA;
-        ++kv->append_launches;
-      }
-    }
-    const int r = release_slot(slot, st);
-    slot = nullptr;
-    n_ids = 0;
-    n_cpy = 0;
-    return r;
-  };
+  ExtendOut& x = kv->ext;
+  x.clear();
   for (int j = 0; j < n_tasks; ++j) {
     const int t = task_ids[j];
     const int c = indptr[j + 1] - indptr[j];
-    if (c == 0) continue;
     auto& pg = kv->pages[t];
+    x.new_lp0.push_back((int32_t)pg.size());
+    x.new_off.push_back((int32_t)x.idx.size());
+    if (c == 0) continue;
     if (last_page_shared(kv, t)) {
-      if ((rc = open_slot()) != TIDE_OK) return rc;
-      if (n_ids == kSlotPageIds || n_cpy == kSlotRecs) {
-        if ((rc = flush()) != TIDE_OK || (rc = open_slot()) != TIDE_OK) return rc;
-      }
       const int32_t old_page = pg.back(), new_page = pop_page(kv);
-      if (cow_out != nullptr) {
-        cow_out->push_back(old_page);
-        cow_out->push_back(new_page);
-      }
-      cpy_src[n_cpy] = old_page;
-      cpy_dst[n_cpy] = new_page;
-      ++n_cpy;
-      idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size() - 1;
-      val[n_ids] = new_page;
-      ++n_ids;
+      x.cpy_src.push_back(old_page);
+      x.cpy_dst.push_back(new_page);
+      x.new_lp0.back() = (int32_t)pg.size() - 1;             // the copy takes the old page's place in the table
+      x.idx.push_back(t * g.max_pages_per_task + (int32_t)pg.size() - 1);
+      x.val.push_back(new_page);
       pg.back() = new_page;
       unref_page(kv, old_page);
     }
     const int new_pages = ceil_div(kv->len[t] + c, g.S) - ceil_div(kv->len[t], g.S);
     for (int k = 0; k < new_pages; ++k) {
-      if ((rc = open_slot()) != TIDE_OK) return rc;
-      if (n_ids == kSlotPageIds) {
-        if ((rc = flush()) != TIDE_OK || (rc = open_slot()) != TIDE_OK) return rc;
-      }
       const int32_t page = pop_page(kv);
-      idx[n_ids] = t * g.max_pages_per_task + (int32_t)pg.size();
-      val[n_ids] = page;
-      ++n_ids;
+      x.idx.push_back(t * g.max_pages_per_task + (int32_t)pg.size());
+      x.val.push_back(page);
       pg.push_back(page);
     }
     kv->len[t] += c;
     kv->used_tokens += c;
   }
-  return flush();
+  return TIDE_OK;
+}
+
+// The private page copies of kv->ext on every layer, in uploads of bounded size.
+static int upload_cow_copies(tide_kv* kv, cudaStream_t st) {
+  const ExtendOut& x = kv->ext;
+  for (size_t done = 0; done < x.cpy_src.size();) {
+    Slot* slot;
+    int rc = acquire_slot(kv, &slot);
+    if (rc != TIDE_OK) return rc;
+    const size_t n = std::min<size_t>(kSlotRecs, x.cpy_src.size() - done);
+    int32_t* h = (int32_t*)(slot->host + 256);
+    std::memcpy(h, x.cpy_src.data() + done, n * 4);
+    std::memcpy(h + n, x.cpy_dst.data() + done, n * 4);
+    if (upload(kv, slot->dev + 256, h, 2 * n * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    const int32_t* d = (const int32_t*)(slot->dev + 256);
+    for (int l = 0; l < kv->cfg.num_layers; ++l) {
+      if (launch_copy_pages(kv->layer_pool(l), d, d + n, (int)n, kv->g.page_bytes, st) != cudaSuccess) return TIDE_ERR_CUDA;
+      ++kv->append_launches;
+    }
+    if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+    done += n;
+  }
+  return TIDE_OK;
+}
+
+// The page-table delta of kv->ext to the device table (a launch of its own), in uploads of bounded size.
+static int upload_table_delta(tide_kv* kv, cudaStream_t st) {
+  const ExtendOut& x = kv->ext;
+  for (size_t done = 0; done < x.idx.size();) {
+    Slot* slot;
+    int rc = acquire_slot(kv, &slot);
+    if (rc != TIDE_OK) return rc;
+    const size_t n = std::min<size_t>(kSlotPageIds, x.idx.size() - done);
+    int32_t* h = (int32_t*)(slot->host + 256);
+    std::memcpy(h, x.idx.data() + done, n * 4);
+    std::memcpy(h + n, x.val.data() + done, n * 4);
+    if (upload(kv, slot->dev + 256, h, 2 * n * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    const int32_t* d = (const int32_t*)(slot->dev + 256);
+    if (launch_table_update(kv->d_table, d, d + n, (int)n, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++kv->append_launches;
+    if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+    done += n;
+  }
+  return TIDE_OK;
+}
+
+// extend_bookkeeping, then the device side: the page-table delta and (with cow_out == nullptr) the private page
+// copies on every layer; otherwise the (old, new) page pairs are handed back and the caller copies (it may have to
+// read the old pages first).
+static int extend_tasks(tide_kv* kv, int32_t n_tasks, const int32_t* task_ids, const int32_t* indptr, cudaStream_t st,
+                        std::vector<int32_t>* cow_out) {
+  int rc = extend_bookkeeping(kv, n_tasks, task_ids, indptr);
+  if (rc != TIDE_OK) return rc;
+  if ((rc = upload_table_delta(kv, st)) != TIDE_OK) return rc;
+  if (cow_out != nullptr) {
+    for (size_t i = 0; i < kv->ext.cpy_src.size(); ++i) {
+      cow_out->push_back(kv->ext.cpy_src[i]);
+      cow_out->push_back(kv->ext.cpy_dst[i]);
+    }
+    return TIDE_OK;
+  }
+  return upload_cow_copies(kv, st);
 }
 
 // Writes the K/V rows of one layer into the LAST indptr[j+1]-indptr[j] positions of task_ids[j] (pure data; the
@@ -571,6 +591,9 @@ static int write_tasks(tide_kv* kv, int32_t layer, int32_t n_tasks, const int32_
       r.pos0 = kv->len[task_ids[j]] - c;
       r.tok0 = indptr[j] - tok_lo;
       r.count = c;
+      r.new_lp0 = INT_MAX;
+      r.new_off = 0;
+      r.pad0 = r.pad1 = 0;
       tok_hi = indptr[j + 1];
     }
     if (n_recs > 0) {
@@ -635,8 +658,56 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
   cudaStream_t st = (cudaStream_t)stream;
   kv->append_launches = 0;
   if (kv->profiling) cudaEventRecord(kv->ev_append[0], st);
-  if ((rc = extend_tasks(kv, n_tasks, task_ids, indptr, st, nullptr)) != TIDE_OK) return rc;
-  if ((rc = write_tasks(kv, 0, n_tasks, task_ids, indptr, new_k, new_v, st)) != TIDE_OK) return rc;
+  if ((rc = extend_bookkeeping(kv, n_tasks, task_ids, indptr)) != TIDE_OK) return rc;
+  if ((rc = upload_cow_copies(kv, st)) != TIDE_OK) return rc;     // a copied page must be in place before it is written
+  int n_recs = 0;
+  for (int j = 0; j < n_tasks; ++j) n_recs += indptr[j + 1] > indptr[j] ? 1 : 0;
+  const ExtendOut& x = kv->ext;
+  if (n_recs <= kSlotRecs && x.idx.size() <= kSlotPageIds) {
+    // The usual case: ONE upload (write records, then the page-table delta) and ONE launch that applies the delta
+    // and scatters the rows; the rows' new pages are read from the delta itself.
+    Slot* slot;
+    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+    AppendRec* recs = (AppendRec*)(slot->host + 256);
+    int r = 0;
+    for (int j = 0; j < n_tasks; ++j) {
+      const int c = indptr[j + 1] - indptr[j];
+      if (c == 0) continue;
+      AppendRec& rec = recs[r++];
+      rec.table_off = task_ids[j] * kv->g.max_pages_per_task;
+      rec.pos0 = kv->len[task_ids[j]] - c;
+      rec.tok0 = indptr[j];
+      rec.count = c;
+      rec.new_lp0 = x.new_lp0[(size_t)j];
+      rec.new_off = x.new_off[(size_t)j];
+      rec.pad0 = rec.pad1 = 0;
+    }
+    const size_t n_ids = x.idx.size();
+    int32_t* h_idx = (int32_t*)(recs + n_recs);
+    std::memcpy(h_idx, x.idx.data(), n_ids * 4);
+    std::memcpy(h_idx + n_ids, x.val.data(), n_ids * 4);
+    const size_t bytes = (size_t)n_recs * sizeof(AppendRec) + 2 * n_ids * 4;
+    if (bytes > 0 && upload(kv, slot->dev + 256, slot->host + 256, bytes, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    AppendParams ap;
+    ap.pool = kv->layer_pool(0);
+    ap.table = kv->d_table;
+    ap.recs = (const AppendRec*)(slot->dev + 256);
+    ap.n_recs = n_recs;
+    ap.n_tokens = indptr[n_tasks];
+    ap.new_k = (const uint16_t*)new_k;
+    ap.new_v = (const uint16_t*)new_v;
+    ap.g = kv->g;
+    ap.table_rw = kv->d_table;
+    ap.upd_idx = (const int32_t*)(ap.recs + n_recs);
+    ap.upd_val = ap.upd_idx + n_ids;
+    ap.n_upd = (int)n_ids;
+    if (launch_append(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++kv->append_launches;
+    if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
+  } else {
+    if ((rc = upload_table_delta(kv, st)) != TIDE_OK) return rc;
+    if ((rc = write_tasks(kv, 0, n_tasks, task_ids, indptr, new_k, new_v, st)) != TIDE_OK) return rc;
+  }
   if (kv->profiling) {
     cudaEventRecord(kv->ev_append[1], st);
     kv->have_append_times = true;
@@ -1206,6 +1277,9 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
     recs[b].pos0 = rows[b].ctx_len - rows[b].q_len;
     recs[b].tok0 = indptr[(size_t)b];
     recs[b].count = rows[b].q_len;
+    recs[b].new_lp0 = INT_MAX;
+    recs[b].new_off = 0;
+    recs[b].pad0 = recs[b].pad1 = 0;
   }
   uint8_t* d_step = kv->ws + kv->lay.off_step;
   const size_t stride = (size_t)kStepSegStride * (size_t)kv->cfg.max_batch_rows;

@@ -1,12 +1,14 @@
 // Internal declarations shared by the host code and the kernels of libtide.so.
 //
 // Physical page layout (private; callers see logical content only):
-//   pool[page][kv_head][K|V][slab = d/64][slot][64 bf16]
-// i.e. for one (page, kv_head) the K block and then the V block, each block made of D/64 slabs of
-// S rows x 128 bytes.  Inside every group of 8 rows the 16-byte chunk c of row r is stored at chunk
-// position c ^ (r & 7) (the 128-byte swizzle of the tensor-core shared-memory layouts).  A plain
-// contiguous bulk copy of a block therefore lands in shared memory ready both for conflict-free
-// ldmatrix and for tcgen05 matrix descriptors, with no tensor map.
+//   pool[page][kv_head][group = slot/8][K|V][slab = d/64][slot%8][64 bf16]
+// i.e. the block of one (page, kv_head) is a run of S/8 groups; a group holds 8 consecutive slots as K then V,
+// each as D/64 slabs of 8 rows x 128 bytes (one 1-KB core-matrix atom of the tensor-core shared-memory
+// layouts).  Inside an atom the 16-byte chunk c of row r is stored at chunk position c ^ r (the 128-byte
+// swizzle).  Consecutive groups - of one page and of the pages copied one after the other into a tile - are a
+// uniform distance apart, so ONE plain contiguous bulk copy of a whole block lands in shared memory ready both
+// for conflict-free ldmatrix and as canonical K-major (K) and MN-major (V) operands of tcgen05 matrix
+// descriptors (stride between 8-key groups = group_bytes, between slabs = 1 KB), with no tensor map.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -26,10 +28,16 @@ constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat fin
 struct Geom {
   int Hq, Hkv, D, S, G;
   int max_pages_per_task;
-  int kblock_bytes;  // one K (or V) block of a (page, head): D*S*2
-  int head_bytes;    // K block + V block
+  int kv_bytes;      // K (or V) part of one 8-slot group: (D/64) * 1024; V sits this far behind K
+  int group_bytes;   // one 8-slot group, K then V: 2 * kv_bytes
+  int head_bytes;    // block of one (page, head): (S/8) * group_bytes
   long long page_bytes;
 };
+
+// Byte offset, inside the block of a (page, head), of the 16-byte chunk c (= d / 8) of slot `slot`; kv = 0 for K, 1 for V.
+__host__ __device__ __forceinline__ int blk_offset(const Geom& g, int slot, int kv, int c) {
+  return (slot >> 3) * g.group_bytes + kv * g.kv_bytes + (c >> 3) * 1024 + (slot & 7) * 128 + (((c & 7) ^ (slot & 7)) << 4);
+}
 
 // One batch row as the kernels see it.  Items of a segment are numbered
 // ((kv_head * n_splits) + split) * n_mtiles + m_tile from item_base.
@@ -98,7 +106,13 @@ struct __align__(16) AppendRec {
   int32_t pos0;       // position in the task of the record's first token
   int32_t tok0;       // index of that token in new_k / new_v
   int32_t count;
+  // When the same launch also applies the page-table delta (AppendParams::upd_*), the table cannot be trusted for
+  // the pages the delta brings: logical pages >= new_lp0 of this record are upd_val[new_off + (lp - new_lp0)].
+  int32_t new_lp0;    // INT_MAX: every page comes from the table
+  int32_t new_off;
+  int32_t pad0, pad1;
 };
+static_assert(sizeof(AppendRec) == 32, "AppendRec layout");
 
 struct AppendParams {
   uint8_t* pool;
@@ -111,6 +125,11 @@ struct AppendParams {
   Geom g;
   const int32_t* dyn = nullptr;   // fixed-grid mode: n_recs = dyn[0], n_tokens = dyn[1]
   int grid_cap_tokens = 0;
+  // page-table delta applied by the same launch: table_rw[upd_idx[i]] = upd_val[i] (n_upd may be 0)
+  int32_t* table_rw = nullptr;
+  const int32_t* upd_idx = nullptr;
+  const int32_t* upd_val = nullptr;
+  int n_upd = 0;
 };
 
 // What tide_attend_decode_static needs of a handle (filled by tide_internal_view in tide_host.cu).
