@@ -123,7 +123,7 @@ def sample_rows(w, n_decode=12):
     return dec + res
 
 
-def build_state(w, torch, tide, seed, picked=()):
+def build_state(w, torch, tide, seed, picked=(), tune=()):
     """Cache with every task's preserved prefix resident, plus this step's device inputs."""
     def dev_bits(a):
         return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda().view(torch.bfloat16)
@@ -131,6 +131,8 @@ def build_state(w, torch, tide, seed, picked=()):
     total_q = int(w.n_new.sum())
     kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task,
                      max_batch_rows=w.B, max_batch_tokens=total_q, free_order=w.free_order)
+    for knob, value in tune:
+        kv.tune(knob, value)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(seed)
     for b in range(w.B):
@@ -303,7 +305,8 @@ def run_ours(args):
     w = inputs.make_workload(args.config, seed=replicas.rank_seed(1000 + args.config, rank), n_tasks=args.tasks, len_div=args.len_div,
                               pool_factor=args.pool_factor)
     picked = sample_rows(w) if rank == 0 else []
-    kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank, picked=picked)
+    tune = [tuple(int(x) for x in kvs.split("=")) for kvs in args.tune]
+    kv, new_k, new_v, q, out, lse = build_state(w, torch, tide, seed=rank, picked=picked, tune=tune)
     rows = tide.rows_array(w.rows())
     ids = np.asarray(w.task, dtype=np.int32)
     indptr = np.concatenate([[0], np.cumsum(w.n_new)]).astype(np.int32)
@@ -355,6 +358,11 @@ def run_ours(args):
     kv.set_profiling(True)
     phases = {"append": [], "decode": [], "tile": [], "merge": []}
     for _ in range(args.steps):
+        # two steps ahead of the measured one keep the device busy while the host enqueues it, so that the phase
+        # events bracket device time only (after a synchronisation the host's own enqueue time would sit inside them)
+        for _ in range(2):
+            step()
+            rollback()
         step()
         ph = kv.phase_ms()
         rollback()
@@ -418,7 +426,7 @@ def run_ours(args):
                        "heads": f"{w.Hq}q/{w.Hkv}kv", "head_dim": w.D, "page_size": w.S,
                        "decode_kv_bytes": dec_bytes, "resume_flops": res_flops,
                        "l2": "inputs larger than L2 (no flush)" if dec_bytes + app_bytes > 2 * 126e6 else "smaller than L2",
-                       "parallelism": f"replicas x{world}", "plan": plan},
+                       "parallelism": f"replicas x{world}", "plan": plan, **({"tune": args.tune} if args.tune else {})},
             "roofline": roof_tensor if use_tensor else roof_hbm,
             "roofline_decode": roof_hbm, "roofline_prefill": roof_tensor,
             "e2e": {"value": dec_bytes_all / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
@@ -798,6 +806,8 @@ def main():
     ap.add_argument("--layers", type=int, default=1,
                     help="> 1 adds a leg that steps this many layers over one page table (planned once, CUDA graph)")
     ap.add_argument("--cpu-budget", type=float, default=20.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--tune", action="append", default=[], metavar="KNOB=VALUE",
+                    help="tide_tune setting for the handle, by the knob's number (see tide_tune_t); may be repeated")
     ap.add_argument("--resident-gb", type=float, default=0.0,
                     help="--config 5 only: GB of KV pool that holds a resident population (150 = the workload as quoted); every "
                          "timed step is then a different batch with releases and admissions in between.  0 = one fixed batch")

@@ -417,6 +417,9 @@ cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s) {
 // ---------------------------------------------------------------------------------------------
 // Log-sum-exp merge of the split partials: one warp per (token, head) row.
 //   LSE = log2 sum_i 2^{LSE_i},  O = sum_i 2^{LSE_i - LSE} O_i;  fixed order, no atomics.
+// The kernel is a chain of dependent loads if written naively (one split after the other), so the partial LSEs
+// are fetched side by side, one per lane, and the partial outputs four splits at a time; the order in which the
+// terms are added is still the order of the splits.
 __global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
   const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
@@ -433,25 +436,48 @@ __global__ void __launch_bounds__(256) merge_kernel(const MergeParams P) {
   auto src_row = [&](int s) -> long long {
     return s < seg.n_splits ? p0 + s * stride : (long long)seg.x_part_base + local + (long long)(s - seg.n_splits) * seg.x_stride;
   };
+  // lane i holds the LSEs of contributions i, i + 32, ... (at most 2 * kMaxSplits = 256 of them)
+  constexpr int kPerLane = 2 * kMaxSplits / 32;
+  float e[kPerLane];
   float mstar = -INFINITY;
-  for (int s = 0; s < n_src; ++s) mstar = fmaxf(mstar, P.part_lse[src_row(s)]);
+#pragma unroll
+  for (int k = 0; k < kPerLane; ++k) {
+    const int s = k * 32 + lane;
+    e[k] = s < n_src ? P.part_lse[src_row(s)] : -INFINITY;
+    mstar = fmaxf(mstar, e[k]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
   const float mu = (mstar == -INFINITY) ? 0.f : mstar;
+#pragma unroll
+  for (int k = 0; k < kPerLane; ++k) e[k] = e[k] == -INFINITY ? 0.f : exp2f(e[k] - mu);   // the contribution's weight
   const int per = P.D / 32;                               // 2 or 4 floats per lane
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   float tot = 0.f;
-  for (int s = 0; s < n_src; ++s) {
-    const long long pr = src_row(s);
-    const float e = P.part_lse[pr];
-    if (e == -INFINITY) continue;
-    const float w = exp2f(e - mu);
-    tot += w;
-    const float* po = P.part_o + pr * P.D + lane * per;
-    if (per == 4) {
-      const float4 v = *reinterpret_cast<const float4*>(po);
-      acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
-    } else {
-      const float2 v = *reinterpret_cast<const float2*>(po);
-      acc[0] += w * v.x; acc[1] += w * v.y;
+  for (int s0 = 0; s0 < n_src; s0 += 4) {
+    float4 v[4];
+    float w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = s0 + u;
+      // weight of contribution s: held by lane s % 32 in its slot s / 32 (kPerLane is small: select, then shuffle)
+      float mine = 0.f;
+#pragma unroll
+      for (int k = 0; k < kPerLane; ++k) if ((s >> 5) == k) mine = e[k];
+      w[u] = s < n_src ? __shfl_sync(0xffffffffu, mine, s & 31) : 0.f;
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (w[u] != 0.f) {
+        const float* po = P.part_o + src_row(s) * P.D + lane * per;
+        if (per == 4) v[u] = *reinterpret_cast<const float4*>(po);
+        else { const float2 t = *reinterpret_cast<const float2*>(po); v[u].x = t.x; v[u].y = t.y; }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (w[u] != 0.f) {
+        tot += w[u];
+        acc[0] += w[u] * v[u].x; acc[1] += w[u] * v[u].y; acc[2] += w[u] * v[u].z; acc[3] += w[u] * v[u].w;
+      }
     }
   }
   const float inv = tot > 0.f ? 1.f / tot : 0.f;

@@ -10,9 +10,9 @@
 // (packed row, key) pair against Hkv*D*4 bytes per key shared by all packed rows.
 //
 // CTA = 12 warps: softmax warpgroups A (warps 0-3) and B (warps 4-7), one thread per row; warp 8 streams tiles of
-// 64 keys, one plain 1-D bulk copy per (page, head) block (blocks are stored as the canonical 128-byte-swizzled
-// core-matrix atoms, K and V of 8 keys side by side, so the blocks of a tile laid one after the other ARE the K-major
-// K operand and the MN-major V operand, a uniform 4 KB between 8-key groups); one lane of warp 9 issues every MMA.
+// 64 keys, one plain 1-D bulk copy per K block and per V block of a (page, head) (blocks are stored as the canonical
+// 128-byte-swizzled core-matrix atoms, so the K blocks of a tile laid one after the other ARE the K-major K operand
+// and the V blocks the MN-major V operand, a uniform 2 KB between 8-key groups); one lane of warp 9 issues every MMA.
 // TMEM (512 columns):
 //   Q_A Q_B   2 x 64   the queries as packed bf16, staged once per item
 //   S_A S_B   2 x 64   fp32 logits of one 64-key tile; P (packed bf16) overwrites the first 32 columns
@@ -38,9 +38,9 @@ constexpr int D = 128;
 constexpr int kTileKeys = 64;
 constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer warp 8, MMA issuer warp 9, two idle warps}
 constexpr int kNumBuf = 6;                          // ring of (K tile, V tile) slots
-constexpr int kKvBytes = (D / 64) * 1024;           // K (or V) of one 8-key group: two 1-KB atoms
-constexpr int kGroupBytes = 2 * kKvBytes;           // one 8-key group: K then V
-constexpr int kSlotBytes = (kTileKeys / 8) * kGroupBytes;   // one 64-key tile, K and V: 32 KB
+constexpr int kGroupBytes = (D / 64) * 1024;        // one 8-key group of a K (or V) tile: two 1-KB atoms
+constexpr int kTileBytes = (kTileKeys / 8) * kGroupBytes;   // one K or V tile of 64 keys: 16 KB
+constexpr int kSlotBytes = 2 * kTileBytes;          // K tile then V tile
 constexpr int kSmemBytes = kNumBuf * kSlotBytes + 1024;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
 constexpr uint32_t kColQ = 0, kColS = 128, kColO = 256;
@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 8) {
-      // ================= producer: one copy per (page, head) block into the ring =================
+      // ================= producer: one copy per K block and per V block of a (page, head) into the ring =================
       if (n_tiles > 0) {
         const int pages_per_tile = kTileKeys / g.S;
         // page ids are fetched 32 logical pages at a time, one per lane, a whole group ahead of their use,
@@ -258,12 +258,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           const int key0 = kv_begin + j * kTileKeys;
           const int npages = min(pages_per_tile, (kv_end - key0 + g.S - 1) / g.S);
           const uint32_t bar = smem_u32(&bars.kv_full[buf]);
-          const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + lane) & 31);
+          // lanes [0, pages_per_tile) fetch the K blocks, lanes [pages_per_tile, 2 * pages_per_tile) the V blocks
+          const int is_v = lane >= pages_per_tile ? 1 : 0, pg = lane - is_v * pages_per_tile;
+          const long long page = __shfl_sync(0xffffffffu, ids_cur, ((j % tiles_per_group) * pages_per_tile + pg) & 31);
           if (lane == 0) mbar_expect_tx(bar, (uint32_t)(npages * g.head_bytes));
           __syncwarp();
-          if (lane < npages)
-            bulk_g2s(smem_base + buf * kSlotBytes + lane * g.head_bytes, P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes,
-                     (uint32_t)g.head_bytes, bar);
+          if (lane < 2 * pages_per_tile && pg < npages)
+            bulk_g2s(smem_base + buf * kSlotBytes + is_v * kTileBytes + pg * g.kblock_bytes,
+                     P.pool + page * g.page_bytes + (long long)kvh * g.head_bytes + is_v * g.kblock_bytes, (uint32_t)g.kblock_bytes, bar);
         }
         if (*abort_flag && lane == 0) {
           // a wait gave up somewhere: do not leave while copies into this CTA's shared memory can still be landing.
@@ -290,7 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
           mma_commit(smem_u32(&bars.s_full[t]));
         };
         auto issue_pv = [&](int t, int j) {
-          const uint32_t vbuf = smem_base + (j % kNumBuf) * kSlotBytes + kKvBytes;
+          const uint32_t vbuf = smem_base + (j % kNumBuf) * kSlotBytes + kTileBytes;
 #pragma unroll
           for (int ks = 0; ks < kTileKeys / 16; ++ks)
             mma_ts(tmem + kColO + t * 128, tmem + kColS + t * 64 + ks * 8, make_desc(vbuf + ks * 2 * kGroupBytes, 1024, kGroupBytes), kIdescPV,
@@ -307,7 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendPa
             // rows of the V tile past the end of the item were not loaded (or hold stale page slots): clear
             // them so that weight 0 times leftover bits cannot produce NaN
             const int first = kv_end - (kv_begin + j * kTileKeys);
-            uint8_t* vgen = smem_gen + (j % kNumBuf) * kSlotBytes + kKvBytes;
+            uint8_t* vgen = smem_gen + (j % kNumBuf) * kSlotBytes + kTileBytes;
             for (int i = lane; i < (kTileKeys - first) * 16; i += 32) {
               const int rr = first + (i >> 4), c = i & 15;     // whole rows are cleared, so the swizzle does not matter
               *reinterpret_cast<uint4*>(vgen + (rr >> 3) * kGroupBytes + (c >> 3) * 1024 + (rr & 7) * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);

@@ -115,6 +115,7 @@ struct tide_kv {
   int items_per_sm = kTargetItemsPerSm;  // work items the planner aims for per SM
   int num_sms = 0;                       // multiprocessors of the handle's device
   long long wait_limit_ns = kWaitLimitNsDefault;   // bound of every wait inside a kernel
+  int umma_tile_keys = 128;              // key-tile size of the tcgen05 kernel: 64 (Q in TMEM) or 128 (Q in shared memory)
   bool drop_first_stage_once = false;    // test hook: armed by tide_tune, consumed by the next attention launch set
   // multi-layer step held between tide_step_begin and the tide_step_layer calls
   uint8_t* h_step = nullptr;   // pinned staging of the step area
@@ -131,6 +132,7 @@ struct tide_kv {
   int host_step_chunks = 0;   // 0 = by size
   bool slots_mapped = false;     // the staging slots' host addresses are valid on the device too
   bool upload_by_kernel = false;
+  bool always_upload_by_kernel = false;   // planning uploads never use the copy engine (tide_tune)
   uint8_t* layer_pool(int layer) const { return pool + (size_t)layer * layer_stride; }
 };
 
@@ -154,9 +156,9 @@ Geom make_geom(const tide_kv_config_t* c) {
   Geom g;
   g.Hq = c->num_q_heads; g.Hkv = c->num_kv_heads; g.D = c->head_dim; g.S = c->page_size; g.G = g.Hq / g.Hkv;
   g.max_pages_per_task = c->max_pages_per_task;
-  g.kv_bytes = (g.D / 64) * 1024;
-  g.group_bytes = 2 * g.kv_bytes;
-  g.head_bytes = (g.S / 8) * g.group_bytes;
+  g.group_bytes = (g.D / 64) * 1024;
+  g.kblock_bytes = (g.S / 8) * g.group_bytes;
+  g.head_bytes = 2 * g.kblock_bytes;
   g.page_bytes = (long long)g.head_bytes * g.Hkv;
   return g;
 }
@@ -237,7 +239,7 @@ int acquire_slot(tide_kv* kv, Slot** out) {
 // Small upload of planning data from a staging slot.  Normally a copy-engine transfer; while a host-buffer step
 // has large copies in flight on other streams it is done by a kernel instead, which does not queue behind them.
 cudaError_t upload(const tide_kv* kv, void* dst, const void* src, size_t bytes, cudaStream_t st) {
-  if (kv->upload_by_kernel) return launch_upload(dst, src, bytes, st);
+  if (kv->upload_by_kernel || (kv->always_upload_by_kernel && kv->slots_mapped)) return launch_upload(dst, src, bytes, st);
   return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
 }
 
@@ -303,7 +305,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
   kv->num_sms = sm_count();
   ok = ok && kv->num_sms > 0;
-  ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess;
+  ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess && attend_umma128_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_step, lay.step_bytes, cudaHostAllocDefault) == cudaSuccess;
@@ -1168,7 +1170,7 @@ static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32
   if (dyn ? kv->cap_umma > 0 : d.items_umma > 0) {
     ap.segs = d.seg_umma; ap.n_segs = (int)d.n_umma; ap.n_items = (int)d.items_umma;
     ap.dyn = dyn ? dyn + kHdrUmmaItems : nullptr; ap.grid_cap = kv->cap_umma;
-    if (launch_attend_umma(ap, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if ((kv->umma_tile_keys == 128 ? launch_attend_umma128(ap, st) : launch_attend_umma(ap, st)) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
   if (events) cudaEventRecord(kv->ev_attend[2], st);
@@ -1513,6 +1515,11 @@ int tide_tune(tide_kv_t* kv, int knob, int64_t value) {
       kv->wait_limit_ns = value * 1000;
       break;
     case TIDE_TUNE_DROP_FIRST_STAGE: kv->drop_first_stage_once = value != 0; break;
+    case TIDE_TUNE_UPLOAD_BY_KERNEL: kv->always_upload_by_kernel = value != 0; break;
+    case TIDE_TUNE_UMMA_TILE_KEYS:
+      if (value != 64 && value != 128) return TIDE_ERR_INVALID_ARG;
+      kv->umma_tile_keys = (int)value;
+      break;
     default: return TIDE_ERR_INVALID_ARG;
   }
   kv->step_valid = false;   // a held plan was made with the old settings

@@ -1,14 +1,15 @@
 // Internal declarations shared by the host code and the kernels of libtide.so.
 //
 // Physical page layout (private; callers see logical content only):
-//   pool[page][kv_head][group = slot/8][K|V][slab = d/64][slot%8][64 bf16]
-// i.e. the block of one (page, kv_head) is a run of S/8 groups; a group holds 8 consecutive slots as K then V,
-// each as D/64 slabs of 8 rows x 128 bytes (one 1-KB core-matrix atom of the tensor-core shared-memory
-// layouts).  Inside an atom the 16-byte chunk c of row r is stored at chunk position c ^ r (the 128-byte
-// swizzle).  Consecutive groups - of one page and of the pages copied one after the other into a tile - are a
-// uniform distance apart, so ONE plain contiguous bulk copy of a whole block lands in shared memory ready both
-// for conflict-free ldmatrix and as canonical K-major (K) and MN-major (V) operands of tcgen05 matrix
-// descriptors (stride between 8-key groups = group_bytes, between slabs = 1 KB), with no tensor map.
+//   pool[page][kv_head][K|V][group = slot/8][slab = d/64][slot%8][64 bf16]
+// i.e. the block of one (page, kv_head) is its K block followed by its V block; each is a run of S/8 groups of 8
+// consecutive slots, a group being D/64 slabs of 8 rows x 128 bytes (one 1-KB core-matrix atom of the
+// tensor-core shared-memory layouts).  Inside an atom the 16-byte chunk c of row r is stored at chunk position
+// c ^ r (the 128-byte swizzle).  Consecutive groups - of one page, and of the K (or V) blocks of several pages
+// copied one after the other into a tile - are a uniform distance apart, so ONE plain contiguous bulk copy of a
+// K or V block (or of both, for ldmatrix users) lands in shared memory ready both for conflict-free ldmatrix and
+// as a canonical K-major (K) or MN-major (V) operand of tcgen05 matrix descriptors (stride between 8-key groups
+// = group_bytes, between slabs = 1 KB), with no tensor map.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -28,15 +29,15 @@ constexpr int kTargetItemsPerSm = 3;   // measured: fewer, longer items beat fin
 struct Geom {
   int Hq, Hkv, D, S, G;
   int max_pages_per_task;
-  int kv_bytes;      // K (or V) part of one 8-slot group: (D/64) * 1024; V sits this far behind K
-  int group_bytes;   // one 8-slot group, K then V: 2 * kv_bytes
-  int head_bytes;    // block of one (page, head): (S/8) * group_bytes
+  int group_bytes;   // one 8-slot group of a K (or V) block: (D/64) * 1024
+  int kblock_bytes;  // the K (or V) block of one (page, head): (S/8) * group_bytes = S*D*2; V sits this far behind K
+  int head_bytes;    // block of one (page, head): K block + V block
   long long page_bytes;
 };
 
 // Byte offset, inside the block of a (page, head), of the 16-byte chunk c (= d / 8) of slot `slot`; kv = 0 for K, 1 for V.
 __host__ __device__ __forceinline__ int blk_offset(const Geom& g, int slot, int kv, int c) {
-  return (slot >> 3) * g.group_bytes + kv * g.kv_bytes + (c >> 3) * 1024 + (slot & 7) * 128 + (((c & 7) ^ (slot & 7)) << 4);
+  return kv * g.kblock_bytes + (slot >> 3) * g.group_bytes + (c >> 3) * 1024 + (slot & 7) * 128 + (((c & 7) ^ (slot & 7)) << 4);
 }
 
 // One batch row as the kernels see it.  Items of a segment are numbered
@@ -157,6 +158,8 @@ cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);
 cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s);
 cudaError_t attend_kernels_init();
 cudaError_t attend_umma_init();
+cudaError_t launch_attend_umma128(const AttendParams& p, cudaStream_t s);
+cudaError_t attend_umma128_init();
 int sm_count();   // multiprocessors of the current device (looked up once per device)
 
 #ifdef __CUDACC__
