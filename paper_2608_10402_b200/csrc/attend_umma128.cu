@@ -480,22 +480,36 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
       const float mu = (m == -INFINITY) ? 0.f : m;
       const uint64_t sl2_2 = pack2(sl2, sl2), nmu_2 = pack2(-mu, -mu);
       uint64_t sp2[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
+      // The exponentials run on the ex2 unit (and, for a share of them, on the FMA and integer pipes), the sums and the
+      // bf16 packing on the FMA and ALU pipes.  A warp issues in order, so the three only overlap if independent work
+      // is next to each other in the instruction stream: the stream is written as a software pipeline over groups of
+      // 8 keys - scaled logits for all groups first, then the exponentials of group g+1 ahead of the sum and the
+      // packing of group g, whose exponentials have had a whole group's time to come back.
+      uint64_t x2[64];
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {                            // P_t over the first 64 columns of S_t, 32 columns (64 keys) at a time
-        uint32_t pk[32];
+      for (int i = 0; i < 64; ++i) x2[i] = fma2(pack2(s[2 * i], s[2 * i + 1]), sl2_2, nmu_2);
+      float e[2][8];
+      auto exp_group = [&](int gidx, float (&eg)[8]) {
 #pragma unroll
-        for (int c = 0; c < 64; c += 8) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            float x0, x1, e0, e1;
-            unpack2(fma2(pack2(s[h * 64 + c + 2 * i], s[h * 64 + c + 2 * i + 1]), sl2_2, nmu_2), x0, x1);
-            if (i < kEmu) poly_exp2_pair(x0, x1, e0, e1);
-            else { e0 = fast_exp2(x0); e1 = fast_exp2(x1); }
-            sp2[i] = add2(sp2[i], pack2(e0, e1));
-            pk[(c >> 1) + i] = pack_bf16(e0, e1);
-          }
+        for (int i = 0; i < 4; ++i) {
+          float x0, x1;
+          unpack2(x2[gidx * 4 + i], x0, x1);
+          if (i < kEmu) poly_exp2_pair(x0, x1, eg[2 * i], eg[2 * i + 1]);
+          else { eg[2 * i] = fast_exp2(x0); eg[2 * i + 1] = fast_exp2(x1); }
         }
-        tmem_st32u(s_addr + h * 32, pk);
+      };
+      uint32_t pk[32];
+      exp_group(0, e[0]);
+#pragma unroll
+      for (int gidx = 0; gidx < 16; ++gidx) {
+        if (gidx + 1 < 16) exp_group(gidx + 1, e[(gidx + 1) & 1]);
+        const float (&eg)[8] = e[gidx & 1];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          sp2[i] = add2(sp2[i], pack2(eg[2 * i], eg[2 * i + 1]));
+          pk[(gidx & 7) * 4 + i] = pack_bf16(eg[2 * i], eg[2 * i + 1]);
+        }
+        if ((gidx & 7) == 7) tmem_st32u(s_addr + (gidx >> 3) * 32, pk);   // P_t over the first 64 columns of S_t, 32 columns (64 keys) at a time
       }
       float sp[8];
 #pragma unroll
