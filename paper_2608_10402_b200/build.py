@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtide.so")
-SOURCES = ["tide_host.cu", "kv_pages.cu", "attend_mma.cu", "attend_umma.cu", "attend_umma128.cu", "attend_umma4.cu", "attend_static.cu"]
+SOURCES = ["tide_host.cu", "kv_pages.cu", "attend_mma.cu", "attend_umma.cu", "attend_umma128.cu", "attend_static.cu"]
 HEADERS = ["tide_internal.h", os.path.join("..", "..", "include", "tide.h")]
 
 

@@ -42,6 +42,10 @@ constexpr uint32_t kColS = 0, kColO = 256;          // S_t at kColS + t*128 (P_t
 #define TIDE_UMMA128_EMU_PAIRS 1                    // of every 4 pairs of exponentials, how many take the polynomial
 #endif
 constexpr int kEmuPairs = TIDE_UMMA128_EMU_PAIRS;
+#ifndef TIDE_UMMA128_P_PARTS
+#define TIDE_UMMA128_P_PARTS 2                      // P_t is handed to the MMA warp in this many parts (2 or 4)
+#endif
+constexpr int kPParts = TIDE_UMMA128_P_PARTS;
 
 // instruction descriptor: fp32 accumulate, bf16 A and B, M = 128, N = 128; bit 16 = B is MN-major
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24) | ((128u >> 3) << 17);
@@ -119,6 +123,14 @@ __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[3
         "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16u(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
   uint32_t u[32];
 #pragma unroll
@@ -174,7 +186,7 @@ struct Bars {
   uint64_t kv_empty[kNumUnits];
   uint64_t q_full;
   uint64_t s_full[2];   // S_t(j) is in TMEM (and every earlier MMA, PV_t(j-1) included, has retired)
-  uint64_t p_full[2];   // P_t(j) is in TMEM
+  uint64_t p_part[2][kPParts];   // part q of P_t(j) (keys [q, q+1) * 128 / kPParts) is in TMEM
   uint64_t o_full[2];   // the last PV_t has retired
   uint64_t mma_done;    // every MMA of the item has retired
 };
@@ -248,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
     mbar_init(smem_u32(&bars.q_full), 256);
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.p_full[t]), 128);
+      for (int q = 0; q < kPParts; ++q) mbar_init(smem_u32(&bars.p_part[t][q]), 128);
       mbar_init(smem_u32(&bars.o_full[t]), 1);
     }
     mbar_init(smem_u32(&bars.mma_done), 1);
@@ -336,12 +348,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
                    desc64(k_lo + (((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), kd_hi), kIdescQK, ks > 0);
           mma_commit(smem_u32(&bars.s_full[t]));
         };
-        auto issue_pv = [&](int t, int j, int slot) {
+        auto issue_pv = [&](int t, int j, int slot, int part) {      // the PV MMAs of part `part` of the keys
           const uint32_t v_lo = vd_lo + slot * kUnitStep;
 #pragma unroll
-          for (int ks = 0; ks < kTileKeys / 16; ++ks)
+          for (int k4 = 0; k4 < kTileKeys / 16 / kPParts; ++k4) {
+            const int ks = part * (kTileKeys / 16 / kPParts) + k4;
             mma_ts(tmem + kColO + t * 128, tmem + kColS + t * 128 + ks * 8, desc64(v_lo + ((ks * 2 * kGroupBytes) >> 4), vd_hi), kIdescPV,
                    (j > 0 || ks > 0) ? 1u : 0u);
+          }
         };
         // operand u of the sequence K0 V0 K1 V1 ... sits in unit u % kNumUnits on its (u / kNumUnits)-th use
         auto wait_full = [&](int slot, int use) {
@@ -370,9 +384,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
           bool k_ready = false;
           for (int t = 0; t < 2; ++t) {
             if (j < t_tiles[t]) {
-              mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag, P.status, P.wait_limit_ns);
-              tc_fence_after();
-              issue_pv(t, j, vslot);
+#pragma unroll
+              for (int q = 0; q < kPParts; ++q) {
+                mbar_wait(smem_u32(&bars.p_part[t][q]), j & 1, abort_flag, P.status, P.wait_limit_ns);
+                tc_fence_after();
+                issue_pv(t, j, vslot, q);
+              }
               if (j + 1 < t_tiles[t]) {
                 if (!k_ready) { wait_full(kslot, kuse); tc_fence_after(); k_ready = true; }
                 issue_qk(t, kslot);                          // overwrites S_t / P_t after PV_t(j), in order
@@ -509,7 +526,19 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
           sp2[i] = add2(sp2[i], pack2(eg[2 * i], eg[2 * i + 1]));
           pk[(gidx & 7) * 4 + i] = pack_bf16(eg[2 * i], eg[2 * i + 1]);
         }
-        if ((gidx & 7) == 7) tmem_st32u(s_addr + (gidx >> 3) * 32, pk);   // P_t over the first 64 columns of S_t, 32 columns (64 keys) at a time
+        // P_t over the first 64 columns of S_t; a part is handed over as soon as it is stored, so that its PV runs
+        // while the exponentials of the later parts are computed (the last part is handed over after the row sum)
+        constexpr int kGroupsPerPart = 16 / kPParts;
+        if ((gidx + 1) % kGroupsPerPart == 0) {
+          const int q = gidx / kGroupsPerPart;
+          if constexpr (kPParts == 2) tmem_st32u(s_addr + q * 32, pk);
+          else tmem_st16u(s_addr + q * 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[(q & 1) * 16]));
+          if (q + 1 < kPParts) {
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars.p_part[t][q]));
+          }
+        }
       }
       float sp[8];
 #pragma unroll
@@ -517,7 +546,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma128_kernel(const Atten
       l = l * alpha + (((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7])));
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars.p_full[t]));
+      mbar_arrive(smem_u32(&bars.p_part[t][kPParts - 1]));
     };
     // tiles j < n_plain end at or before the first row's limit: every key of theirs is visible to every row
     const int n_plain = min(my_tiles, max(0, (t_min_limit[t] - kv_begin) / kTileKeys));

@@ -305,7 +305,7 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
   kv->num_sms = sm_count();
   ok = ok && kv->num_sms > 0;
-  ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess && attend_umma128_init() == cudaSuccess && attend_umma4_init() == cudaSuccess;
+  ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess && attend_umma128_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_step, lay.step_bytes, cudaHostAllocDefault) == cudaSuccess;
@@ -1170,9 +1170,7 @@ static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32
   if (dyn ? kv->cap_umma > 0 : d.items_umma > 0) {
     ap.segs = d.seg_umma; ap.n_segs = (int)d.n_umma; ap.n_items = (int)d.items_umma;
     ap.dyn = dyn ? dyn + kHdrUmmaItems : nullptr; ap.grid_cap = kv->cap_umma;
-    const cudaError_t e = kv->umma_tile_keys == 4 ? launch_attend_umma4(ap, st)
-                          : kv->umma_tile_keys == 128 ? launch_attend_umma128(ap, st) : launch_attend_umma(ap, st);
-    if (e != cudaSuccess) return TIDE_ERR_CUDA;
+    if ((kv->umma_tile_keys == 128 ? launch_attend_umma128(ap, st) : launch_attend_umma(ap, st)) != cudaSuccess) return TIDE_ERR_CUDA;
     ++launches;
   }
   if (events) cudaEventRecord(kv->ev_attend[2], st);
@@ -1519,7 +1517,7 @@ int tide_tune(tide_kv_t* kv, int knob, int64_t value) {
     case TIDE_TUNE_DROP_FIRST_STAGE: kv->drop_first_stage_once = value != 0; break;
     case TIDE_TUNE_UPLOAD_BY_KERNEL: kv->always_upload_by_kernel = value != 0; break;
     case TIDE_TUNE_UMMA_TILE_KEYS:
-      if (value != 64 && value != 128 && value != 4) return TIDE_ERR_INVALID_ARG;
+      if (value != 64 && value != 128) return TIDE_ERR_INVALID_ARG;
       kv->umma_tile_keys = (int)value;
       break;
     default: return TIDE_ERR_INVALID_ARG;

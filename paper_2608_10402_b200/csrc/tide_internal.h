@@ -160,8 +160,6 @@ cudaError_t attend_kernels_init();
 cudaError_t attend_umma_init();
 cudaError_t launch_attend_umma128(const AttendParams& p, cudaStream_t s);
 cudaError_t attend_umma128_init();
-cudaError_t launch_attend_umma4(const AttendParams& p, cudaStream_t s);
-cudaError_t attend_umma4_init();
 int sm_count();   // multiprocessors of the current device (looked up once per device)
 
 #ifdef __CUDACC__

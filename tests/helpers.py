@@ -34,12 +34,14 @@ def from_dev(t):
     return t.cpu().numpy().view(np.uint16)
 
 
-def gpu_fill(w, kv_bits, nk, nv, indptr, tide, torch, max_batch_tokens=None):
+def gpu_fill(w, kv_bits, nk, nv, indptr, tide, torch, max_batch_tokens=None, tune=()):
     """The same sequence of calls on the CUDA library."""
     total_q = int(w.n_new.sum())
     kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task,
                      max_batch_rows=max(w.B, 1), max_batch_tokens=max_batch_tokens or max(total_q, 1),
                      free_order=w.free_order)
+    for knob, value in tune:
+        kv.tune(knob, value)
     for b in range(w.B):
         kv.alloc(int(w.task[b]))
     for b in range(w.B):

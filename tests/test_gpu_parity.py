@@ -20,11 +20,11 @@ def env():
     return tide, torch
 
 
-def run_workload(w, tide, torch, full_oracle=True, seed=0):
+def run_workload(w, tide, torch, full_oracle=True, seed=0, tune=()):
     kv_bits = [w.task_kv(b) for b in range(w.B)]
     q_bits = np.concatenate([w.task_q(b) for b in range(w.B)])
     c, indptr, nk, nv = H.oracle_fill(w, kv_bits)
-    kv = H.gpu_fill(w, kv_bits, nk, nv, indptr, tide, torch)
+    kv = H.gpu_fill(w, kv_bits, nk, nv, indptr, tide, torch, tune=tune)
     H.compare_bookkeeping(w, c, kv)
     H.compare_cache(w, c, kv)
     total_q = q_bits.shape[0]
@@ -55,6 +55,13 @@ def test_config1_tiny_ctb_step(env):
 def test_reduced_configs_full_oracle(env, index, n_tasks, len_div):
     tide, torch = env
     run_workload(inputs.make_workload(index, n_tasks=n_tasks, len_div=len_div), tide, torch)
+
+
+@pytest.mark.parametrize("index,n_tasks,len_div", [(3, 12, 8), (4, 6, 16), (5, 16, 16)])
+def test_the_64_key_tcgen05_kernel_matches_too(env, index, n_tasks, len_div):
+    # the append-prefill kernel with 64-key tiles (Q in TMEM) stays selectable next to the default 128-key one
+    tide, torch = env
+    run_workload(inputs.make_workload(index, n_tasks=n_tasks, len_div=len_div), tide, torch, tune=[(tide.TUNE_UMMA_TILE_KEYS, 64)])
 
 
 def _single_row_case(tide, torch, Hq, Hkv, D, S, n, L, q_bits, k_bits, v_bits, scale, free_seed=0):
