@@ -250,8 +250,8 @@ typedef enum {
                                   /* tcgen05 kernel, >= 17 (default 17)                                            */
   TIDE_TUNE_WAIT_LIMIT_US = 5,    /* time limit of every wait inside a kernel, microseconds (default 2 000 000)    */
   TIDE_TUNE_UMMA_TILE_KEYS = 7,   /* key-tile size of the tcgen05 kernel: 64 or 128                                */
-  TIDE_TUNE_UPLOAD_BY_KERNEL = 8, /* non-zero: the small planning uploads of every call are done by a kernel that   */
-                                  /* reads the pinned staging slot instead of by the copy engine                   */
+  TIDE_TUNE_UPLOAD_BY_KERNEL = 8, /* the small planning uploads of every call are done by a kernel that reads the   */
+                                  /* pinned, device-mapped staging slot (default 1) or by the copy engine (0)       */
   TIDE_TUNE_DROP_FIRST_STAGE = 6  /* test hook, non-zero arms it for the NEXT attention call only: in work item 0   */
                                   /* of each attention kernel of that call the K/V producer leaves out (its part   */
                                   /* of) the first stage, so the wait for that stage runs out and the time-out     */
