@@ -76,8 +76,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
   const int qi_lo = r_lo / g.G, qi_hi = r_hi / g.G;
   const int hd_lo = kvh * g.G + (r_lo - qi_lo * g.G), hd_hi = kvh * g.G + (r_hi - qi_hi * g.G);
 
-  if (kv_end <= kv_begin) {
-    // nothing visible in this split (only possible when n_splits > 1): neutral partials
+  if (kv_end <= kv_begin && seg.partial != 2) {
+    // nothing visible in this split (only possible when n_splits > 1): neutral partials.  (A segment whose last split
+    // merges walks the normal path with zero stages instead, so that it is counted.)
     if (warp < kConsumerWarps && (lane & 3) == 0 && (!DECODE || warp == 0)) {
       if (v_lo) P.part_lse[seg.part_base + (split * seg.n + qi_lo) * g.Hq + hd_lo] = -INFINITY;
       if (v_hi) P.part_lse[seg.part_base + (split * seg.n + qi_hi) * g.Hq + hd_hi] = -INFINITY;
@@ -381,6 +382,53 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
 #pragma unroll
         for (int d = 0; d < DSEG; d += 4) *reinterpret_cast<float4*>(dst + d) = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
         if ((t & 7) == 0) P.part_lse[prow] = e2;
+      }
+    }
+    // A split decode-style row merges its own partials: every split counts itself in once its partials are written
+    // (fence, barrier, one atomic per CTA); the CTA that counts last reads all splits' partials - in split order, so
+    // the result does not depend on which one came last - and writes the row.  The counter goes back to zero for the
+    // next launch.  This removes the merge launch, and with it a dependent chain of loads, from decode-only steps.
+    if (seg.partial == 2) {
+      __shared__ int s_is_last;
+      __threadfence();
+      named_bar_sync(1, kConsumerWarps * 32);
+      if (t == 0) {
+        int* ctr = P.merge_ctr + seg.x_part_base + kvh;
+        const int done = atomicAdd(ctr, 1);
+        s_is_last = done == seg.n_splits - 1 ? 1 : 0;
+        if (s_is_last) *ctr = 0;
+      }
+      named_bar_sync(1, kConsumerWarps * 32);
+      if (s_is_last && r < R) {
+        __threadfence();
+        const int qi = r / g.G, hd = kvh * g.G + (r - qi * g.G);
+        const long long stride = (long long)seg.n * g.Hq;                       // partial rows per split
+        const long long p0 = seg.part_base + (long long)qi * g.Hq + hd;         // this (token, head) in split 0
+        float mstar = -INFINITY;
+        for (int sp = 0; sp < seg.n_splits; ++sp) mstar = fmaxf(mstar, __ldcg(P.part_lse + p0 + sp * stride));
+        const float mu = (mstar == -INFINITY) ? 0.f : mstar;
+        float acc[DSEG];
+#pragma unroll
+        for (int d = 0; d < DSEG; ++d) acc[d] = 0.f;
+        float tot = 0.f;
+        for (int sp = 0; sp < seg.n_splits; ++sp) {
+          const float e = __ldcg(P.part_lse + p0 + sp * stride);
+          if (e == -INFINITY) continue;
+          const float w = exp2f(e - mu);
+          tot += w;
+          const float4* po = reinterpret_cast<const float4*>(P.part_o + (p0 + sp * stride) * D + d0);
+#pragma unroll
+          for (int d = 0; d < DSEG; d += 4) {
+            const float4 v = __ldcg(po + (d >> 2));
+            acc[d] += w * v.x; acc[d + 1] += w * v.y; acc[d + 2] += w * v.z; acc[d + 3] += w * v.w;
+          }
+        }
+        const float inv = tot > 0.f ? 1.f / tot : 0.f;
+        const long long orow = (long long)(seg.q_off + qi) * g.Hq + hd;
+        uint32_t* dst = reinterpret_cast<uint32_t*>(P.out + orow * D + d0);
+#pragma unroll
+        for (int d = 0; d < DSEG; d += 2) dst[d >> 1] = pack_bf16(acc[d] * inv, acc[d + 1] * inv);
+        if (P.lse != nullptr && (t & 7) == 0) P.lse[orow] = (tot > 0.f ? mstar + log2f(tot) : -INFINITY) * kLn2;
       }
     }
   }

@@ -34,7 +34,7 @@ constexpr size_t kHostChunkBytes = 64u << 20;      // transfer bytes per group f
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t off_status, off_table, off_old_row, off_step, off_meta, off_part_o, off_part_lse, off_stage_k, off_stage_v,
+  size_t off_status, off_table, off_old_row, off_merge_ctr, off_step, off_meta, off_part_o, off_part_lse, off_stage_k, off_stage_v,
       off_stage_q, off_stage_out, off_stage_lse, total;
   size_t slot_bytes;
   size_t step_bytes;      // held plan of a multi-layer step: write records, then segments
@@ -53,6 +53,7 @@ struct PlanDev {
 struct PlanHost {
   std::vector<Segment> seg_dec, seg_tile, seg_umma, seg_merge;
   long long items_dec = 0, items_tile = 0, items_umma = 0, merge_rows = 0;
+  long long fused_rows = 0;   // rows whose partials are merged by the decode kernel itself (not part of merge_rows)
   size_t n_all() const { return seg_dec.size() + seg_tile.size() + seg_umma.size() + seg_merge.size(); }
 };
 
@@ -86,6 +87,7 @@ struct tide_kv {
   int* d_status = nullptr;
   float* d_part_o = nullptr;
   float* d_part_lse = nullptr;
+  int* d_merge_ctr = nullptr;   // finished-split counters of the segments whose last split merges (zero between launches)
   Slot slots[kSlots];
   int next_slot = 0;
   int* h_status = nullptr;  // pinned
@@ -170,6 +172,7 @@ Layout make_layout(const tide_kv_config_t* c, const Geom& g) {
   L.off_status = off; off += 256;
   L.off_table = off; off = align_up(off + (size_t)c->max_tasks * c->max_pages_per_task * 4, 256);
   L.off_old_row = off; off = align_up(off + (size_t)c->max_pages_per_task * 4 + 64, 256);   // row + one page pair
+  L.off_merge_ctr = off; off = align_up(off + (size_t)kStepSegStride * c->max_batch_rows * g.Hkv * 4, 256);   // finished-split counters
   // step area: 256-byte header of counts | write records | four segment arrays of max_batch_rows entries each
   L.step_seg_off = align_up(256 + (size_t)c->max_batch_rows * sizeof(AppendRec), 256);
   L.step_bytes = align_up(L.step_seg_off + (size_t)(4 * kStepSegStride * c->max_batch_rows) * sizeof(Segment), 256);
@@ -303,11 +306,13 @@ int tide_kv_create(const tide_kv_config_t* cfg, tide_kv_t** out) {
   kv->d_old_row = (int32_t*)(kv->ws + lay.off_old_row);
   kv->d_part_o = (float*)(kv->ws + lay.off_part_o);
   kv->d_part_lse = (float*)(kv->ws + lay.off_part_lse);
+  kv->d_merge_ctr = (int*)(kv->ws + lay.off_merge_ctr);
   bool ok = cudaGetDevice(&kv->device) == cudaSuccess;
   kv->num_sms = sm_count();
   ok = ok && kv->num_sms > 0;
   ok = ok && attend_kernels_init() == cudaSuccess && attend_umma_init() == cudaSuccess && attend_umma128_init() == cudaSuccess;
   ok = ok && cudaMemset(kv->d_status, 0, 256) == cudaSuccess;
+  ok = ok && cudaMemset(kv->d_merge_ctr, 0, (size_t)kStepSegStride * cfg->max_batch_rows * g.Hkv * 4) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_status, 64, cudaHostAllocDefault) == cudaSuccess;
   ok = ok && cudaHostAlloc((void**)&kv->h_step, lay.step_bytes, cudaHostAllocDefault) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&kv->ev_step, cudaEventDisableTiming) == cudaSuccess;
@@ -1073,7 +1078,9 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
   std::stable_sort(P.seg_umma.begin(), P.seg_umma.end(), heavier);
   P.seg_merge.clear();
   P.merge_rows = 0;
+  P.fused_rows = 0;
   long long part_cursor = 0;
+  int32_t ctr_cursor = 0;
   std::vector<Segment*> merged;                              // segments with rows to merge, in merge_base order
   for (auto* v : {&P.seg_dec, &P.seg_tile, &P.seg_umma}) {
     long long base = 0;
@@ -1087,6 +1094,12 @@ static int build_plan(tide_kv* kv, int32_t n_rows, const tide_row_t* rows, bool 
         if (s.x_n_splits == -2) {                            // a shared range: it has no output rows of its own
           groups[(size_t)s.x_part_base].part_base = s.part_base;
           groups[(size_t)s.x_part_base].n_splits = s.n_splits;
+        } else if (v == &P.seg_dec && s.partial == 0 && s.x_n_splits == 0) {
+          // a plain split decode-style row: the split that finishes last merges the partials inside the decode kernel
+          s.partial = 2;
+          s.x_part_base = ctr_cursor;
+          ctr_cursor += g.Hkv;
+          P.fused_rows += (long long)s.n * g.Hq;
         } else {
           s.merge_base = (int32_t)P.merge_rows;
           P.merge_rows += (long long)s.n * g.Hq;
@@ -1149,6 +1162,7 @@ static int launch_plan(tide_kv* kv, int32_t layer, const PlanDev& d, const int32
   ap.scale_log2e = scale * 1.4426950408889634f;
   ap.status = kv->d_status;
   ap.g = kv->g;
+  ap.merge_ctr = kv->d_merge_ctr;
   ap.wait_limit_ns = kv->wait_limit_ns;
   ap.debug_drop_first_stage = kv->drop_first_stage_once ? 1 : 0;
   kv->drop_first_stage_once = false;
@@ -1218,7 +1232,7 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   if ((rc = release_slot(slot, st)) != TIDE_OK) return rc;
   kv->last_decode_items = pd.items_dec;
   kv->last_prefill_items = pd.items_tile + pd.items_umma;
-  kv->last_merge_rows = pd.merge_rows;
+  kv->last_merge_rows = pd.merge_rows + P.fused_rows;
   kv->last_launches = launches + kv->append_launches;
   kv->append_launches = 0;
   return TIDE_OK;
@@ -1304,7 +1318,7 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
   kv->step_valid = true;
   kv->last_decode_items = P.items_dec;
   kv->last_prefill_items = P.items_tile + P.items_umma;
-  kv->last_merge_rows = P.merge_rows;
+  kv->last_merge_rows = P.merge_rows + P.fused_rows;
   return TIDE_OK;
 }
 
@@ -1453,6 +1467,8 @@ int tide_status(tide_kv_t* kv, void* stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
   const int code = *kv->h_status;
   if (code != 0) {
+    // a launch that was cut short may have left finished-split counters behind
+    if (cudaMemsetAsync(kv->d_merge_ctr, 0, (size_t)kStepSegStride * kv->cfg.max_batch_rows * kv->g.Hkv * 4, st) != cudaSuccess) return TIDE_ERR_CUDA;
     if (cudaMemsetAsync(kv->d_status, 0, sizeof(int), st) != cudaSuccess) return TIDE_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
   }

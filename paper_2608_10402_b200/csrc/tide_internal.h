@@ -58,7 +58,9 @@ struct __align__(16) Segment {
   // member's own range starts behind it (origin), both write partials, and the member's merge takes both.
   int32_t causal;      // query i sees keys [0, p + i * causal + 1): 1 for a task's own tokens, 0 for a shared range
   int32_t origin;      // first key of the range this segment covers (split s starts at origin + s * chunk)
-  int32_t partial;     // 1: write partials even when n_splits == 1 (another segment contributes to the same rows)
+  int32_t partial;     // 1: write partials even when n_splits == 1 (another segment contributes to the same rows);
+                       // 2: a split decode-style segment whose last-finishing split merges the partials itself
+                       //    (AttendParams::merge_ctr[x_part_base + kv_head] counts the finished splits)
   int32_t x_part_base; // the other contribution to this segment's rows: first partial row of token 0's head 0 ...
   int32_t x_n_splits;  // ... its number of splits (0 = none) ...
   int32_t x_stride;    // ... and the distance in rows between its consecutive splits
@@ -83,6 +85,7 @@ struct AttendParams {
   // kernel reads n_items = dyn[0] and n_segs = dyn[1] from device memory; CTAs beyond n_items leave at once.
   const int32_t* dyn = nullptr;
   int grid_cap = 0;
+  int* merge_ctr = nullptr;   // per (segment with partial == 2, kv head): splits finished so far; zero between launches
   long long wait_limit_ns = kWaitLimitNsDefault;   // bound of every wait inside the kernel
   // Test hook for the bounded waits (never set in normal use): in work item 0 the producer leaves out its part
   // of the first stage, so the consumers' wait for that stage runs out and the time-out path executes.
