@@ -30,9 +30,9 @@ sys.path.insert(0, ROOT)
 METRIC = "mixed resume batch: KV-read GB/s vs HBM peak; append-prefill TFLOP/s vs peak"
 # DRAM traffic per unit of algorithmic work, from the ncu captures summarised under profiles/ (reduced cases,
 # scaled by the units one launch processes): decode kernel dram bytes / algorithmic KV bytes; tcgen05 kernel
-# dram bytes per flop of resume-row attention.
-NCU_DECODE_TRAFFIC_RATIO = 1.011
-NCU_UMMA_DRAM_BYTES_PER_FLOP = 348.6e6 / 863.8e9
+# dram bytes / algorithmic bytes of its launch (K and V of every resume row once + Q + O).
+NCU_DECODE_TRAFFIC_RATIO = 1.012
+NCU_UMMA_TRAFFIC_RATIO = 350.2e6 / 359.2e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -93,7 +93,7 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------------------
-def rooflines(peaks, dec_bytes, dec_ms, res_flops, tile_ms, timed_ms):
+def rooflines(peaks, dec_bytes, dec_ms, res_flops, tile_ms, timed_ms, res_bytes):
     """The two roofline objects of a step: decode rows against the measured HBM copy rate (algorithmic KV bytes of
     the decode rows / device time of the decode-style kernel) and resume rows against the measured bf16 tensor rate
     (algorithmic flops / device time of the tile kernels; the burst peak unless the timed region is over a second)."""
@@ -102,8 +102,8 @@ def rooflines(peaks, dec_bytes, dec_ms, res_flops, tile_ms, timed_ms):
     tpeak = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
     roof_tensor = {"bound": "tensor", "kernel": "attend tile kernel (resume rows)",
                    "achieved": res_flops / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0,
-                   "peak": tpeak, "unit": "TFLOP/s", "traffic": res_flops * NCU_UMMA_DRAM_BYTES_PER_FLOP,
-                   "traffic_note": "dram read+write bytes of a reduced-case ncu capture scaled by flops (see profiles/)",
+                   "peak": tpeak, "unit": "TFLOP/s", "traffic": res_bytes * NCU_UMMA_TRAFFIC_RATIO,
+                   "traffic_note": "ncu dram read+write of a reduced case / its algorithmic bytes (K,V of the resume rows once + Q + O), scaled (see profiles/)",
                    "peak_source": f"{peaks['_source']} ({'sustained' if sustained else 'burst'} bf16)"}
     roof_tensor["frac"] = roof_tensor["achieved"] / tpeak
     roof_hbm = {"bound": "hbm", "kernel": "attend decode kernel (decode rows)",
@@ -410,8 +410,10 @@ def run_ours(args):
         reduced = args.tasks is not None or args.len_div != 1 or args.pool_factor is not None
         n_app = int(w.n_new.sum())
         app_bytes = 2 * w.kv_bytes_per_token() * n_app
+        res_rows = w.n_new > 1
+        res_bytes = int(w.kv_bytes_per_token() * int(w.ctx[res_rows].sum()) + int(w.n_new[res_rows].sum()) * w.Hq * w.D * 4)
         use_tensor, roof_hbm, roof_tensor = rooflines(peaks, dec_bytes, ph_ms["decode"], res_flops, ph_ms["tile"],
-                                                      step_ms * args.steps)
+                                                      step_ms * args.steps, res_bytes)
         line = {
             "metric": METRIC, "value": kv_gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -661,7 +663,7 @@ def run_long_horizon(args):
     kv.set_profiling(True)
     sampler = ClockSampler(local)
     sampler.start()
-    tot = {"ms": 0.0, "append": 0.0, "decode": 0.0, "tile": 0.0, "merge": 0.0, "dec_bytes": 0.0, "flops": 0.0, "tokens": 0, "launches": 0}
+    tot = {"ms": 0.0, "append": 0.0, "decode": 0.0, "tile": 0.0, "merge": 0.0, "dec_bytes": 0.0, "flops": 0.0, "res_bytes": 0.0, "tokens": 0, "launches": 0}
     step_ms_list, last = [], None
     for it in range(warmup + steps):
         batch, n_new, indptr, nk, nv, q, rows = make_batch()
@@ -688,6 +690,7 @@ def run_long_horizon(args):
                 tot[k] += ph[k]
             tot["dec_bytes"] += HKV * D * 4 * sum(r[2] for r in rows if r[1] == 1)
             tot["flops"] += 4 * D * HQ * sum(r[1] * (r[2] - r[1]) + r[1] * (r[1] + 1) // 2 for r in rows if r[1] > 1)
+            tot["res_bytes"] += sum(HKV * D * 4 * r[2] + r[1] * HQ * D * 4 for r in rows if r[1] > 1)
             tot["tokens"] += int(indptr[-1])
             tot["launches"] += kv.last_plan()["kernel_launches"]
             last = (rows, indptr, q, out, lse)
@@ -752,7 +755,8 @@ def run_long_horizon(args):
         [tot["ms"], tot["decode"], tot["tile"], tot["append"], tot["merge"], e2e_ms],
         [tot["dec_bytes"], tot["flops"], tot["e2e_dec_bytes"]], world, dist, "cuda")
     if rank == 0:
-        use_tensor, roof_hbm, roof_tensor = rooflines(peaks, tot["dec_bytes"], tot["decode"], tot["flops"], tot["tile"], tot["ms"])
+        use_tensor, roof_hbm, roof_tensor = rooflines(peaks, tot["dec_bytes"], tot["decode"], tot["flops"], tot["tile"], tot["ms"],
+                                                      tot["res_bytes"])
         line = {
             "metric": METRIC, "value": replicas.whole_job_rate(dec_bytes_all, dec_ms) / 1e9, "unit": "GB/s", "n_gpus": world,
             "steps": steps, "warmup": warmup, "ms_per_step": step_ms / steps, "higher_is_better": True, "scaling": "weak",
