@@ -32,7 +32,7 @@ METRIC = "mixed resume batch: KV-read GB/s vs HBM peak; append-prefill TFLOP/s v
 # scaled by the units one launch processes): decode kernel dram bytes / algorithmic KV bytes; tcgen05 kernel
 # dram bytes / algorithmic bytes of its launch (K and V of every resume row once + Q + O).
 NCU_DECODE_TRAFFIC_RATIO = 1.012
-NCU_UMMA_TRAFFIC_RATIO = 350.2e6 / 359.2e6
+NCU_UMMA_TRAFFIC_RATIO = 1155.1e6 / 1153.2e6     # one-pass capture of the full-size mixed batch
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -103,7 +103,7 @@ def rooflines(peaks, dec_bytes, dec_ms, res_flops, tile_ms, timed_ms, res_bytes)
     roof_tensor = {"bound": "tensor", "kernel": "attend tile kernel (resume rows)",
                    "achieved": res_flops / (tile_ms * 1e-3) / 1e12 if tile_ms > 0 else 0.0,
                    "peak": tpeak, "unit": "TFLOP/s", "traffic": res_bytes * NCU_UMMA_TRAFFIC_RATIO,
-                   "traffic_note": "ncu dram read+write of a reduced case / its algorithmic bytes (K,V of the resume rows once + Q + O), scaled (see profiles/)",
+                   "traffic_note": "ncu dram read+write of one full-size launch / its algorithmic bytes (K,V of the resume rows once + Q + O), times this launch's algorithmic bytes (see profiles/)",
                    "peak_source": f"{peaks['_source']} ({'sustained' if sustained else 'burst'} bf16)"}
     roof_tensor["frac"] = roof_tensor["achieved"] / tpeak
     roof_hbm = {"bound": "hbm", "kernel": "attend decode kernel (decode rows)",
