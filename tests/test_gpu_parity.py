@@ -64,6 +64,13 @@ def test_the_64_key_tcgen05_kernel_matches_too(env, index, n_tasks, len_div):
     run_workload(inputs.make_workload(index, n_tasks=n_tasks, len_div=len_div), tide, torch, tune=[(tide.TUNE_UMMA_TILE_KEYS, 64)])
 
 
+def test_planning_uploads_through_the_copy_engine_match_too(env):
+    # by default the small planning uploads are done by a kernel that reads the mapped staging slot; the copy-engine
+    # path stays selectable and must give the same pages, cache bits and outputs
+    tide, torch = env
+    run_workload(inputs.make_workload(3, n_tasks=12, len_div=8), tide, torch, tune=[(tide.TUNE_UPLOAD_BY_KERNEL, 0)])
+
+
 def _single_row_case(tide, torch, Hq, Hkv, D, S, n, L, q_bits, k_bits, v_bits, scale, free_seed=0):
     pages = (L + S - 1) // S + 3
     kv = tide.TideKV(Hq, Hkv, D, S, pages, 2, pages, 4, max(n, 4),
