@@ -252,6 +252,9 @@ typedef enum {
   TIDE_TUNE_UMMA_TILE_KEYS = 7,   /* key-tile size of the tcgen05 kernel: 64 or 128                                */
   TIDE_TUNE_UPLOAD_BY_KERNEL = 8, /* the small planning uploads of every call are done by a kernel that reads the   */
                                   /* pinned, device-mapped staging slot (default 1) or by the copy engine (0)       */
+  TIDE_TUNE_INLINE_DESCRIPTORS = 9, /* small appends (<= 128 rows, <= 256 new pages) and decode-only batches of up  */
+                                  /* to 128 rows carry their descriptors in the launch's own parameters, so that  */
+                                  /* nothing is uploaded before the kernel (default 1); 0: always upload           */
   TIDE_TUNE_DROP_FIRST_STAGE = 6  /* test hook, non-zero arms it for the NEXT attention call only: in work item 0   */
                                   /* of each attention kernel of that call the K/V producer leaves out (its part   */
                                   /* of) the first stage, so the wait for that stage runs out and the time-out     */

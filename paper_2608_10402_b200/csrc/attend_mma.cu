@@ -30,7 +30,7 @@ struct MmaCfg {
 };
 
 template <int D, bool DECODE>
-__global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const AttendParams P) {
+__device__ __forceinline__ void attend_mma_body(const AttendParams& P, const Segment* __restrict__ segs) {
   constexpr int KS = D / 16;                 // k-steps of Q.K^T
   constexpr int NT = D / 8;                  // n-tiles of O
   constexpr int STEP_KB = DECODE ? 1 : 4;    // 16-key blocks per softmax step of one warp
@@ -54,8 +54,8 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
     if (item >= P.dyn[0]) return;
     n_segs = P.dyn[1];
   }
-  const int si = find_segment(n_segs, item, [&](int i) { return P.segs[i].item_base; });
-  const Segment seg = P.segs[si];
+  const int si = find_segment(n_segs, item, [&](int i) { return segs[i].item_base; });
+  const Segment seg = segs[si];
   int local = item - seg.item_base;
   const int m_tile = local % seg.n_mtiles;
   local /= seg.n_mtiles;
@@ -434,6 +434,17 @@ __global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const Att
   }
 }
 
+template <int D, bool DECODE>
+__global__ void __launch_bounds__(kAttendThreads, 2) attend_mma_kernel(const AttendParams P) {
+  attend_mma_body<D, DECODE>(P, P.segs);
+}
+
+// Decode-style items whose row descriptors travel in the kernel's parameters (small decode-only batches).
+template <int D>
+__global__ void __launch_bounds__(kAttendThreads, 2) attend_decode_inline_kernel(const __grid_constant__ AttendInline PI) {
+  attend_mma_body<D, true>(PI.p, PI.segs);
+}
+
 cudaError_t attend_kernels_init() {
   cudaError_t e;
   e = cudaFuncSetAttribute(attend_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<128>::kSmemBytes);
@@ -443,7 +454,19 @@ cudaError_t attend_kernels_init() {
   e = cudaFuncSetAttribute(attend_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<64>::kSmemBytes);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attend_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<64>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_decode_inline_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<128>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attend_decode_inline_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MmaCfg<64>::kSmemBytes);
   return e;
+}
+
+cudaError_t launch_attend_decode_inline(const AttendInline& pi, cudaStream_t s) {
+  const int grid = pi.p.n_items;
+  if (grid <= 0) return cudaSuccess;
+  if (pi.p.g.D == 128) attend_decode_inline_kernel<128><<<grid, kAttendThreads, MmaCfg<128>::kSmemBytes, s>>>(pi);
+  else attend_decode_inline_kernel<64><<<grid, kAttendThreads, MmaCfg<64>::kSmemBytes, s>>>(pi);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s) {

@@ -51,15 +51,16 @@ constexpr int kAppendLoadsInFlight = 8;    // 16-byte loads a lane has in flight
 // pages that delta brings are then taken from the delta itself, not from the table (no ordering between thread
 // blocks is needed).
 template <int CPL>
-__global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_kernel(const AppendParams P) {
+__device__ __forceinline__ void append_scatter_body(const AppendParams& P, const AppendRec* __restrict__ recs,
+                                                    const int32_t* __restrict__ upd_idx, const int32_t* __restrict__ upd_val) {
   __shared__ int32_t s_tok0[kAppendMaxRecsSmem];
   const int n_recs = P.dyn ? P.dyn[0] : P.n_recs;
   const int n_tokens = P.dyn ? P.dyn[1] : P.n_tokens;
   for (int i = blockIdx.x * kAppendThreads + threadIdx.x; i < P.n_upd; i += gridDim.x * kAppendThreads)
-    P.table_rw[P.upd_idx[i]] = P.upd_val[i];
+    P.table_rw[upd_idx[i]] = upd_val[i];
   const bool in_smem = n_recs <= kAppendMaxRecsSmem;
   if (in_smem) {
-    for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = P.recs[i].tok0;
+    for (int i = threadIdx.x; i < n_recs; i += blockDim.x) s_tok0[i] = recs[i].tok0;
     __syncthreads();
   }
   const Geom& g = P.g;
@@ -74,12 +75,12 @@ __global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_kernel(const
   auto locate = [&](int tok, int& slot) -> uint8_t* {
     int r;
     if (in_smem) r = find_segment(n_recs, tok, [&](int i) { return s_tok0[i]; });
-    else r = find_segment(n_recs, tok, [&](int i) { return P.recs[i].tok0; });
-    const AppendRec rec = P.recs[r];
+    else r = find_segment(n_recs, tok, [&](int i) { return recs[i].tok0; });
+    const AppendRec rec = recs[r];
     const int pos = rec.pos0 + (tok - rec.tok0);
     const int lp = pos / g.S;
     slot = pos - lp * g.S;
-    const long long page = lp >= rec.new_lp0 ? P.upd_val[rec.new_off + (lp - rec.new_lp0)] : P.table[rec.table_off + lp];
+    const long long page = lp >= rec.new_lp0 ? upd_val[rec.new_off + (lp - rec.new_lp0)] : P.table[rec.table_off + lp];
     return P.pool + page * g.page_bytes;
   };
   // chunk c of a token: source address and offset inside the page
@@ -127,22 +128,53 @@ __global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_kernel(const
   }
 }
 
+template <int CPL>
+__global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_kernel(const AppendParams P) {
+  append_scatter_body<CPL>(P, P.recs, P.upd_idx, P.upd_val);
+}
+
+// The same with the records and the table delta inside the kernel's parameters (small appends: nothing to upload).
+template <int CPL>
+__global__ void __launch_bounds__(kAppendThreads, 3) append_scatter_inline_kernel(const __grid_constant__ AppendInline PI) {
+  append_scatter_body<CPL>(PI.p, PI.recs, PI.upd, PI.upd + PI.p.n_upd);
+}
+
+static unsigned append_grid(const AppendParams& p, int& cpl) {
+  const int tokens = p.dyn ? p.grid_cap_tokens : p.n_tokens;
+  const int cpt = 2 * p.g.Hkv * (p.g.D / 8);
+  cpl = cpt % 32 == 0 ? cpt / 32 : 0;
+  if (!(cpl == 1 || cpl == 2 || cpl == 4 || cpl == 8)) cpl = 0;
+  const int tok_per_round = cpl ? kAppendLoadsInFlight / cpl : 1;
+  long long blocks = ((long long)std::max(tokens, 1) + kAppendWarps * tok_per_round - 1) / (kAppendWarps * tok_per_round);
+  const long long cap = (long long)sm_count() * 3;   // the resident blocks; each warp loops over rounds beyond this
+  return (unsigned)std::max<long long>(1, std::min(blocks, cap));
+}
+
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
   const int tokens = p.dyn ? p.grid_cap_tokens : p.n_tokens;
   if (tokens <= 0 && p.n_upd <= 0) return cudaSuccess;
-  const int cpt = 2 * p.g.Hkv * (p.g.D / 8);
-  const int cpl = cpt % 32 == 0 ? cpt / 32 : 0;
-  const int tok_per_round = (cpl == 1 || cpl == 2 || cpl == 4 || cpl == 8) ? kAppendLoadsInFlight / cpl : 1;
-  long long blocks = ((long long)std::max(tokens, 1) + kAppendWarps * tok_per_round - 1) / (kAppendWarps * tok_per_round);
-  const long long cap = (long long)sm_count() * 3;   // the resident blocks; each warp loops over rounds beyond this
-  blocks = std::max<long long>(1, std::min(blocks, cap));
-  const dim3 grid((unsigned)blocks);
+  int cpl;
+  const dim3 grid(append_grid(p, cpl));
   switch (cpl) {
     case 1: append_scatter_kernel<1><<<grid, kAppendThreads, 0, s>>>(p); break;
     case 2: append_scatter_kernel<2><<<grid, kAppendThreads, 0, s>>>(p); break;
     case 4: append_scatter_kernel<4><<<grid, kAppendThreads, 0, s>>>(p); break;
     case 8: append_scatter_kernel<8><<<grid, kAppendThreads, 0, s>>>(p); break;
     default: append_scatter_kernel<0><<<grid, kAppendThreads, 0, s>>>(p); break;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append_inline(const AppendInline& pi, cudaStream_t s) {
+  if (pi.p.n_tokens <= 0 && pi.p.n_upd <= 0) return cudaSuccess;
+  int cpl;
+  const dim3 grid(append_grid(pi.p, cpl));
+  switch (cpl) {
+    case 1: append_scatter_inline_kernel<1><<<grid, kAppendThreads, 0, s>>>(pi); break;
+    case 2: append_scatter_inline_kernel<2><<<grid, kAppendThreads, 0, s>>>(pi); break;
+    case 4: append_scatter_inline_kernel<4><<<grid, kAppendThreads, 0, s>>>(pi); break;
+    case 8: append_scatter_inline_kernel<8><<<grid, kAppendThreads, 0, s>>>(pi); break;
+    default: append_scatter_inline_kernel<0><<<grid, kAppendThreads, 0, s>>>(pi); break;
   }
   return cudaGetLastError();
 }

@@ -87,6 +87,8 @@ struct tide_kv {
   int* d_status = nullptr;
   float* d_part_o = nullptr;
   float* d_part_lse = nullptr;
+  AppendInline append_inline;   // host images of the launches that carry their descriptors
+  AttendInline attend_inline;
   int* d_merge_ctr = nullptr;   // finished-split counters of the segments whose last split merges (zero between launches)
   Slot slots[kSlots];
   int next_slot = 0;
@@ -134,6 +136,7 @@ struct tide_kv {
   int host_step_chunks = 0;   // 0 = by size
   bool slots_mapped = false;     // the staging slots' host addresses are valid on the device too
   bool upload_by_kernel = false;
+  bool inline_descriptors = true;         // small appends and decode-only batches carry their descriptors in the launch
   bool always_upload_by_kernel = true;    // planning uploads by a kernel reading the mapped staging slot, not by the copy engine
                                           // (measured on a 64-row decode step: 157 -> 147 us; tide_tune can switch it off)
   uint8_t* layer_pool(int layer) const { return pool + (size_t)layer * layer_stride; }
@@ -671,12 +674,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
   int n_recs = 0;
   for (int j = 0; j < n_tasks; ++j) n_recs += indptr[j + 1] > indptr[j] ? 1 : 0;
   const ExtendOut& x = kv->ext;
-  if (n_recs <= kSlotRecs && x.idx.size() <= kSlotPageIds) {
-    // The usual case: ONE upload (write records, then the page-table delta) and ONE launch that applies the delta
-    // and scatters the rows; the rows' new pages are read from the delta itself.
-    Slot* slot;
-    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
-    AppendRec* recs = (AppendRec*)(slot->host + 256);
+  auto fill_recs = [&](AppendRec* recs) {
     int r = 0;
     for (int j = 0; j < n_tasks; ++j) {
       const int c = indptr[j + 1] - indptr[j];
@@ -690,6 +688,35 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
       rec.new_off = x.new_off[(size_t)j];
       rec.pad0 = rec.pad1 = 0;
     }
+  };
+  if (kv->inline_descriptors && n_recs <= kInlineRecs && x.idx.size() <= (size_t)kInlineUpd) {
+    // A small append: the write records and the page-table delta travel in the launch's own parameters, so there
+    // is nothing to upload and ONE launch does everything.
+    AppendInline& pi = kv->append_inline;
+    fill_recs(pi.recs);
+    const size_t n_ids = x.idx.size();
+    std::memcpy(pi.upd, x.idx.data(), n_ids * 4);
+    std::memcpy(pi.upd + n_ids, x.val.data(), n_ids * 4);
+    AppendParams& ap = pi.p;
+    ap = AppendParams();
+    ap.pool = kv->layer_pool(0);
+    ap.table = kv->d_table;
+    ap.n_recs = n_recs;
+    ap.n_tokens = indptr[n_tasks];
+    ap.new_k = (const uint16_t*)new_k;
+    ap.new_v = (const uint16_t*)new_v;
+    ap.g = kv->g;
+    ap.table_rw = kv->d_table;
+    ap.n_upd = (int)n_ids;
+    if (launch_append_inline(pi, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    ++kv->append_launches;
+  } else if (n_recs <= kSlotRecs && x.idx.size() <= kSlotPageIds) {
+    // The usual case: ONE upload (write records, then the page-table delta) and ONE launch that applies the delta
+    // and scatters the rows; the rows' new pages are read from the delta itself.
+    Slot* slot;
+    if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
+    AppendRec* recs = (AppendRec*)(slot->host + 256);
+    fill_recs(recs);
     const size_t n_ids = x.idx.size();
     int32_t* h_idx = (int32_t*)(recs + n_recs);
     std::memcpy(h_idx, x.idx.data(), n_ids * 4);
@@ -1222,6 +1249,42 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
   if (P.n_all() * sizeof(Segment) + 256 > kv->lay.slot_bytes) return TIDE_ERR_WORKSPACE;
 
   cudaStream_t st = (cudaStream_t)stream;
+  if (kv->inline_descriptors && P.seg_tile.empty() && P.seg_umma.empty() && P.seg_merge.empty() &&
+      P.seg_dec.size() <= (size_t)kInlineSegs) {
+    // A small decode-only batch: the row descriptors travel in the decode launch's own parameters (no upload).
+    AttendInline& pi = kv->attend_inline;
+    std::copy(P.seg_dec.begin(), P.seg_dec.end(), pi.segs);
+    AttendParams& ap = pi.p;
+    ap = AttendParams();
+    ap.pool = kv->layer_pool(layer);
+    ap.table = page_table ? page_table : kv->d_table;
+    ap.n_segs = (int)P.seg_dec.size();
+    ap.n_items = (int)P.items_dec;
+    ap.q = (const uint16_t*)q;
+    ap.out = (uint16_t*)out;
+    ap.lse = lse;
+    ap.part_o = kv->d_part_o;
+    ap.part_lse = kv->d_part_lse;
+    ap.scale_log2e = scale * 1.4426950408889634f;
+    ap.status = kv->d_status;
+    ap.g = kv->g;
+    ap.merge_ctr = kv->d_merge_ctr;
+    ap.wait_limit_ns = kv->wait_limit_ns;
+    ap.debug_drop_first_stage = kv->drop_first_stage_once ? 1 : 0;
+    kv->drop_first_stage_once = false;
+    if (kv->profiling) cudaEventRecord(kv->ev_attend[0], st);
+    if (launch_attend_decode_inline(pi, st) != cudaSuccess) return TIDE_ERR_CUDA;
+    if (kv->profiling) {
+      for (int i = 1; i <= 3; ++i) cudaEventRecord(kv->ev_attend[i], st);
+      kv->have_attend_times = true;
+    }
+    kv->last_decode_items = P.items_dec;
+    kv->last_prefill_items = 0;
+    kv->last_merge_rows = P.fused_rows;
+    kv->last_launches = 1 + kv->append_launches;
+    kv->append_launches = 0;
+    return TIDE_OK;
+  }
   Slot* slot;
   if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
   const PlanDev pd = pack_plan(P, (Segment*)(slot->host + 256), (const Segment*)(slot->dev + 256), 0);
@@ -1533,6 +1596,7 @@ int tide_tune(tide_kv_t* kv, int knob, int64_t value) {
       break;
     case TIDE_TUNE_DROP_FIRST_STAGE: kv->drop_first_stage_once = value != 0; break;
     case TIDE_TUNE_UPLOAD_BY_KERNEL: kv->always_upload_by_kernel = value != 0; break;
+    case TIDE_TUNE_INLINE_DESCRIPTORS: kv->inline_descriptors = value != 0; break;
     case TIDE_TUNE_UMMA_TILE_KEYS:
       if (value != 64 && value != 128) return TIDE_ERR_INVALID_ARG;
       kv->umma_tile_keys = (int)value;

@@ -136,6 +136,22 @@ struct AppendParams {
   int n_upd = 0;
 };
 
+// Small batches carry their descriptors in the launch itself: a decode-only batch of up to kInlineSegs rows, and an
+// append of up to kInlineRecs records with up to kInlineUpd new page-table entries, need no upload before the kernel
+// (the kernels read them from their own parameter space), which takes one launch each out of a decode step.
+constexpr int kInlineSegs = 128;
+constexpr int kInlineRecs = 128;
+constexpr int kInlineUpd = 256;
+struct AttendInline {
+  AttendParams p;                  // p.segs is not used
+  Segment segs[kInlineSegs];
+};
+struct AppendInline {
+  AppendParams p;                  // p.recs, p.upd_idx, p.upd_val are not used
+  AppendRec recs[kInlineRecs];
+  int32_t upd[2 * kInlineUpd];     // p.n_upd table indices, then p.n_upd values
+};
+
 // What tide_attend_decode_static needs of a handle (filled by tide_internal_view in tide_host.cu).
 struct StaticView {
   Geom g;
@@ -156,6 +172,8 @@ cudaError_t launch_copy_pages(uint8_t* pool, const int32_t* src, const int32_t* 
 cudaError_t launch_read(const uint8_t* pool, const int32_t* table_row, int pos0, int len, uint16_t* out_k,
                         uint16_t* out_v, const Geom& g, cudaStream_t s);
 cudaError_t launch_attend_decode(const AttendParams& p, cudaStream_t s);
+cudaError_t launch_attend_decode_inline(const AttendInline& p, cudaStream_t s);   // p.p.n_segs <= kInlineSegs, exact grid
+cudaError_t launch_append_inline(const AppendInline& p, cudaStream_t s);
 cudaError_t launch_attend_tile(const AttendParams& p, cudaStream_t s);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t s);
 cudaError_t launch_attend_umma(const AttendParams& p, cudaStream_t s);

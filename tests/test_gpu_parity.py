@@ -64,6 +64,14 @@ def test_the_64_key_tcgen05_kernel_matches_too(env, index, n_tasks, len_div):
     run_workload(inputs.make_workload(index, n_tasks=n_tasks, len_div=len_div), tide, torch, tune=[(tide.TUNE_UMMA_TILE_KEYS, 64)])
 
 
+def test_small_batches_with_uploaded_descriptors_match_too(env):
+    # by default a small append and a small decode-only batch carry their descriptors in the launch's parameters; with
+    # that turned off they are uploaded like those of large batches, and the results must be the same
+    tide, torch = env
+    run_workload(inputs.make_workload(2, n_tasks=12, len_div=8), tide, torch, tune=[(tide.TUNE_INLINE_DESCRIPTORS, 0)])
+    run_workload(inputs.make_workload(1), tide, torch, tune=[(tide.TUNE_INLINE_DESCRIPTORS, 0)])
+
+
 def test_planning_uploads_through_the_copy_engine_match_too(env):
     # by default the small planning uploads are done by a kernel that reads the mapped staging slot; the copy-engine
     # path stays selectable and must give the same pages, cache bits and outputs
