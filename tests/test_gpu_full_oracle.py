@@ -1,9 +1,11 @@
 """Every query of a full-size batch against the float64 oracle, element by element (not a sample).
 
-The mixed multi-turn text resume batch at its full size (128 tasks, 96 decode rows, 32 resume rows of 200..2000
-appended tokens over contexts of 2k..32k) costs the oracle about two minutes on 16 host cores and runs with the
-routine GPU tests.  The multimodal resume batch (32 rows of 1000..3000 image tokens over contexts up to 64k)
-costs it about a quarter of an hour and runs when TIDE_FULL_ORACLE_ALL=1.  With TIDE_REPORT_DIR set, a per-row
+The decode-only batch (64 rows) costs the oracle a second, and the mixed multi-turn text resume batch at its full
+size (128 tasks, 96 decode rows, 32 resume rows of 200..2000 appended tokens over contexts of 2k..32k) about three
+minutes on 16 host cores: both run with the routine GPU tests.  The long-horizon stress batch (230 decode rows and
+26 resume rows of 500..4000 tokens over contexts up to 128k) costs it another three minutes and the multimodal
+resume batch (32 rows of 1000..3000 image tokens over contexts up to 64k) 23: they run when
+TIDE_FULL_ORACLE_ALL=1.  With TIDE_REPORT_DIR set, a per-row
 table (worst error / tolerance, largest absolute error, relative Frobenius error, LSE error) is written there as
 full_oracle_config<k>.md; profiles/ holds the committed copies.
 
@@ -21,7 +23,7 @@ from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
 
-CASES = [3] + ([4] if os.environ.get("TIDE_FULL_ORACLE_ALL") == "1" else [])
+CASES = [2, 3] + ([4, 5] if os.environ.get("TIDE_FULL_ORACLE_ALL") == "1" else [])
 
 
 @pytest.mark.parametrize("index", CASES)
