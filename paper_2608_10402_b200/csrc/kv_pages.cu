@@ -147,13 +147,7 @@ static unsigned append_grid(const AppendParams& p, int& cpl) {
   const int tok_per_round = cpl ? kAppendLoadsInFlight / cpl : 1;
   long long blocks = ((long long)std::max(tokens, 1) + kAppendWarps * tok_per_round - 1) / (kAppendWarps * tok_per_round);
   const long long cap = (long long)sm_count() * 3;   // the resident blocks; each warp loops over rounds beyond this
-  if (blocks > cap) {
-    // as many blocks as give every one of them the same number of rounds: a last round that only a few blocks
-    // take part in runs at the latency of a round all the same
-    const long long rounds = (blocks + cap - 1) / cap;
-    blocks = (blocks + rounds - 1) / rounds;
-  }
-  return (unsigned)std::max<long long>(1, blocks);
+  return (unsigned)std::max<long long>(1, std::min(blocks, cap));
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t s) {
