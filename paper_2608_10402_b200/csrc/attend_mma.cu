@@ -174,6 +174,22 @@ __device__ __forceinline__ void attend_mma_body(const AttendParams& P, const Seg
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
   const float sl2 = P.scale_log2e;
 
+  // Decode items: a warp reads the same 16 slots of every stage, so the offsets of its ldmatrix rows inside a stage
+  // are fixed for the whole item (two per K n-tile, four for V; the others are 1 KB further on).
+  uint32_t dk_off[2][2] = {{0u, 0u}, {0u, 0u}}, dv_off[4] = {0u, 0u, 0u, 0u};
+  if (DECODE) {
+    const int koff = warp * 16;
+    const uint32_t page_off = (uint32_t)((koff / g.S) * g.head_bytes);
+    const int row0 = koff % g.S;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int x = 0; x < 2; ++x) dk_off[nt][x] = page_off + (uint32_t)blk_offset(g, row0 + nt * 8 + (lane & 7), 0, x * 4 + (lane >> 3));
+    const int vrow = row0 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+    for (int y = 0; y < 4; ++y) dv_off[y] = page_off + (uint32_t)blk_offset(g, vrow, 1, y * 2 + (lane >> 4));
+  }
+
   for (int st = 0; st < n_st; ++st) {
     const int slot = st % kStages;
     mbar_wait(smem_u32(&s_full[slot]), (st / kStages) & 1, abort_flag, P.status, P.wait_limit_ns);
@@ -198,7 +214,8 @@ __device__ __forceinline__ void attend_mma_body(const AttendParams& P, const Seg
 #pragma unroll
             for (int k2 = 0; k2 < KS / 2; ++k2) {
               uint32_t b0, b1, b2, b3;
-              ldsm_x4(pbase + blk_offset(g, slot_row, 0, k2 * 4 + (lane >> 3)), b0, b1, b2, b3);
+              if (DECODE) ldsm_x4(stage + dk_off[nt][k2 & 1] + (k2 >> 1) * 1024, b0, b1, b2, b3);
+              else ldsm_x4(pbase + blk_offset(g, slot_row, 0, k2 * 4 + (lane >> 3)), b0, b1, b2, b3);
               mma_bf16(acc, qa[2 * k2], b0, b1);
               mma_bf16(acc, qa[2 * k2 + 1], b2, b3);
             }
@@ -277,7 +294,8 @@ __device__ __forceinline__ void attend_mma_body(const AttendParams& P, const Seg
 #pragma unroll
           for (int n2 = 0; n2 < NT / 2; ++n2) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4_t(vbase + blk_offset(g, vrow, 1, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
+            if (DECODE) ldsm_x4_t(stage + dv_off[n2 & 3] + (n2 >> 2) * 1024, b0, b1, b2, b3);
+            else ldsm_x4_t(vbase + blk_offset(g, vrow, 1, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
             mma_bf16(o[2 * n2], pa, b0, b1);
             mma_bf16(o[2 * n2 + 1], pa, b2, b3);
           }
