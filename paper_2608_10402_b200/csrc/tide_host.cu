@@ -18,6 +18,7 @@
 
 using namespace tide;
 
+
 namespace {
 
 constexpr int kSlots = 8;                    // staging ring depth
@@ -592,7 +593,7 @@ static int write_tasks(tide_kv* kv, int32_t layer, int32_t n_tasks, const int32_
     Slot* slot;
     if ((rc = acquire_slot(kv, &slot)) != TIDE_OK) return rc;
     AppendRec* recs = (AppendRec*)(slot->host + 256);
-    int n_recs = 0, tok_lo = -1, tok_hi = -1;
+    int n_recs = 0, tok_lo = -1, tok_hi = -1, grp_cursor = 0;
     for (; j < n_tasks && n_recs < kSlotRecs; ++j) {
       const int c = indptr[j + 1] - indptr[j];
       if (c == 0) continue;
@@ -604,7 +605,8 @@ static int write_tasks(tide_kv* kv, int32_t layer, int32_t n_tasks, const int32_
       r.count = c;
       r.new_lp0 = INT_MAX;
       r.new_off = 0;
-      r.pad0 = r.pad1 = 0;
+      r.grp0 = grp_cursor; r.pad1 = 0;
+      grp_cursor += ((r.pos0 & 7) + r.count + 7) >> 3;
       tok_hi = indptr[j + 1];
     }
     if (n_recs > 0) {
@@ -675,7 +677,7 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
   for (int j = 0; j < n_tasks; ++j) n_recs += indptr[j + 1] > indptr[j] ? 1 : 0;
   const ExtendOut& x = kv->ext;
   auto fill_recs = [&](AppendRec* recs) {
-    int r = 0;
+    int r = 0, grp_cursor = 0;
     for (int j = 0; j < n_tasks; ++j) {
       const int c = indptr[j + 1] - indptr[j];
       if (c == 0) continue;
@@ -686,7 +688,8 @@ int tide_kv_append(tide_kv_t* kv, int32_t layer, int32_t n_tasks, const int32_t*
       rec.count = c;
       rec.new_lp0 = x.new_lp0[(size_t)j];
       rec.new_off = x.new_off[(size_t)j];
-      rec.pad0 = rec.pad1 = 0;
+      rec.grp0 = grp_cursor; rec.pad1 = 0;
+      grp_cursor += ((rec.pos0 & 7) + rec.count + 7) >> 3;
     }
   };
   if (kv->inline_descriptors && n_recs <= kInlineRecs && x.idx.size() <= (size_t)kInlineUpd) {
@@ -1352,6 +1355,7 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
   hdr[kHdrUmmaItems] = (int32_t)P.items_umma; hdr[kHdrUmmaItems + 1] = (int32_t)P.seg_umma.size();
   hdr[kHdrMergeRows] = (int32_t)P.merge_rows; hdr[kHdrMergeRows + 1] = (int32_t)P.seg_merge.size();
   AppendRec* recs = (AppendRec*)(kv->h_step + 256);
+  int grp_cursor = 0;
   for (int b = 0; b < n_rows; ++b) {
     recs[b].table_off = rows[b].task * g.max_pages_per_task;
     recs[b].pos0 = rows[b].ctx_len - rows[b].q_len;
@@ -1359,7 +1363,8 @@ int tide_step_begin(tide_kv_t* kv, int32_t n_rows, const tide_row_t* rows, void*
     recs[b].count = rows[b].q_len;
     recs[b].new_lp0 = INT_MAX;
     recs[b].new_off = 0;
-    recs[b].pad0 = recs[b].pad1 = 0;
+    recs[b].grp0 = grp_cursor; recs[b].pad1 = 0;
+    grp_cursor += ((recs[b].pos0 & 7) + recs[b].count + 7) >> 3;
   }
   uint8_t* d_step = kv->ws + kv->lay.off_step;
   const size_t stride = (size_t)kStepSegStride * (size_t)kv->cfg.max_batch_rows;

@@ -114,7 +114,9 @@ struct __align__(16) AppendRec {
   // the pages the delta brings: logical pages >= new_lp0 of this record are upd_val[new_off + (lp - new_lp0)].
   int32_t new_lp0;    // INT_MAX: every page comes from the table
   int32_t new_off;
-  int32_t pad0, pad1;
+  int32_t grp0;       // 8-slot groups of the page blocks that the records before this one touch (a record touches
+                      // ((pos0 & 7) + count + 7) / 8 of them): the append kernel's unit of work
+  int32_t pad1;
 };
 static_assert(sizeof(AppendRec) == 32, "AppendRec layout");
 
