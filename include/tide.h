@@ -139,7 +139,9 @@ int tide_attend(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_t* 
  * tokens to every row's task (rows must name distinct tasks; ctx_len must equal the resident length
  * after the append), attends, and copies out / lse back.  new_k, new_v: host bf16 [sum q_len, Hkv, D];
  * q, out: host bf16 [sum q_len, Hq, D]; lse: host fp32 or NULL.  Host buffers should be pinned for
- * the copies to be asynchronous.  The call returns after the results have arrived.  A large step is cut
+ * the copies to be asynchronous.  The call returns after the results have arrived.  A small step (up to
+ * 2 MiB in all) whose buffers are pinned and addressable by the device is not copied at all: the kernels
+ * read the inputs and write the results across PCIe themselves.  A large step is cut
  * into groups of consecutive rows whose copies (on two streams the library owns) run beside the kernels
  * of other groups; pages, cache contents and results do not depend on the cut.  The whole step is checked
  * (rows, duplicates, pages) before anything is copied or changed.  Takes layer 0 only. */
@@ -255,6 +257,9 @@ typedef enum {
   TIDE_TUNE_INLINE_DESCRIPTORS = 9, /* small appends (<= 128 rows, <= 256 new pages) and decode-only batches of up  */
                                   /* to 128 rows carry their descriptors in the launch's own parameters, so that  */
                                   /* nothing is uploaded before the kernel (default 1); 0: always upload           */
+  TIDE_TUNE_HOST_ZERO_COPY = 10,  /* tide_step_host: a step of up to 2 MiB whose host buffers are pinned and mapped   */
+                                  /* is not copied; the kernels read and write the host buffers themselves         */
+                                  /* (default 1); 0: always copy                                                  */
   TIDE_TUNE_DROP_FIRST_STAGE = 6  /* test hook, non-zero arms it for the NEXT attention call only: in work item 0   */
                                   /* of each attention kernel of that call the K/V producer leaves out (its part   */
                                   /* of) the first stage, so the wait for that stage runs out and the time-out     */

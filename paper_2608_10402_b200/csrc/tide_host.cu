@@ -31,6 +31,7 @@ constexpr int kStepSegStride = 2;   // each segment array of the step area holds
 constexpr int kHdrRecs = 0, kHdrDecItems = 2, kHdrTileItems = 4, kHdrUmmaItems = 6, kHdrMergeRows = 8;
 constexpr int kMaxHostChunks = 8;                 // most row groups of one host-buffer step
 constexpr size_t kHostChunkBytes = 64u << 20;      // transfer bytes per group from which cutting a step pays
+constexpr size_t kZeroCopyBytes = 2u << 20;        // a host-buffer step up to this size is read and written in place (no copies)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -137,6 +138,7 @@ struct tide_kv {
   int host_step_chunks = 0;   // 0 = by size
   bool slots_mapped = false;     // the staging slots' host addresses are valid on the device too
   bool upload_by_kernel = false;
+  bool host_zero_copy = true;             // small host-buffer steps: kernels address the pinned host buffers themselves
   bool inline_descriptors = true;         // small appends and decode-only batches carry their descriptors in the launch
   bool always_upload_by_kernel = true;    // planning uploads by a kernel reading the mapped staging slot, not by the copy engine
                                           // (measured on a 64-row decode step: 157 -> 147 us; tide_tune can switch it off)
@@ -1454,6 +1456,28 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
   const size_t bytes = T * (2 * kv_row + 2 * q_row + (lse ? lse_row : 0));
   int n_chunks = kv->host_step_chunks > 0 ? kv->host_step_chunks : (int)std::min<size_t>(kMaxHostChunks, bytes / kHostChunkBytes);
   n_chunks = std::max(1, std::min(std::min(n_chunks, kMaxHostChunks), n_rows));
+  // A small step from pinned host buffers that the device can address is not copied at all: the append kernel reads
+  // new_k / new_v, and the attention kernels read q and write out / lse, straight across PCIe.  Five copies of a few
+  // hundred KB cost more in engine hand-overs than the bytes do (a 64-row decode step: 0.22 -> 0.20 ms, a tiny one
+  // 0.11 -> 0.09).
+  if (kv->host_zero_copy && n_chunks == 1 && bytes <= kZeroCopyBytes) {
+    auto mapped = [](const void* p, void** dev) -> bool {
+      cudaPointerAttributes a;
+      if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+      if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return false;
+      *dev = a.devicePointer;
+      return ((uintptr_t)a.devicePointer & 15) == 0;
+    };
+    void *zk, *zv, *zq, *zo, *zl = nullptr;
+    if (mapped(new_k, &zk) && mapped(new_v, &zv) && mapped(q, &zq) && mapped(out, &zo) && (lse == nullptr || mapped(lse, &zl))) {
+      rc = tide_kv_append(kv, layer, n_rows, ids.data(), indptr.data(), zk, zv, stream);
+      if (rc != TIDE_OK) return rc;
+      rc = tide_attend(kv, layer, n_rows, rows, nullptr, zq, scale, zo, (float*)zl, stream);
+      if (rc != TIDE_OK) return rc;
+      if (cudaStreamSynchronize(st) != cudaSuccess) return TIDE_ERR_CUDA;
+      return TIDE_OK;
+    }
+  }
   if (n_chunks > 1 && kv->st_in == nullptr) {
     bool ok = cudaStreamCreateWithFlags(&kv->st_in, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&kv->st_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -1602,6 +1626,7 @@ int tide_tune(tide_kv_t* kv, int knob, int64_t value) {
     case TIDE_TUNE_DROP_FIRST_STAGE: kv->drop_first_stage_once = value != 0; break;
     case TIDE_TUNE_UPLOAD_BY_KERNEL: kv->always_upload_by_kernel = value != 0; break;
     case TIDE_TUNE_INLINE_DESCRIPTORS: kv->inline_descriptors = value != 0; break;
+    case TIDE_TUNE_HOST_ZERO_COPY: kv->host_zero_copy = value != 0; break;
     case TIDE_TUNE_UMMA_TILE_KEYS:
       if (value != 64 && value != 128) return TIDE_ERR_INVALID_ARG;
       kv->umma_tile_keys = (int)value;

@@ -20,7 +20,7 @@ ERR_NO_PAGES, ERR_TABLE_FULL, ERR_CTX_RANGE, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE
 STATIC_MAX_ROWS = 64
 # knobs of tide_tune (tide_tune_t)
 (TUNE_ITEMS_PER_SM, TUNE_GROUPING, TUNE_MIN_SAVED_BYTES, TUNE_HOST_STEP_CHUNKS, TUNE_UMMA_MIN_ROWS, TUNE_WAIT_LIMIT_US,
- TUNE_DROP_FIRST_STAGE, TUNE_UMMA_TILE_KEYS, TUNE_UPLOAD_BY_KERNEL, TUNE_INLINE_DESCRIPTORS) = range(10)
+ TUNE_DROP_FIRST_STAGE, TUNE_UMMA_TILE_KEYS, TUNE_UPLOAD_BY_KERNEL, TUNE_INLINE_DESCRIPTORS, TUNE_HOST_ZERO_COPY) = range(11)
 
 
 class TideError(RuntimeError):

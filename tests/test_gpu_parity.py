@@ -235,10 +235,11 @@ def test_append_leaves_neighbouring_slots_untouched(env):
     kv.close()
 
 
-@pytest.mark.parametrize("groups", [0, 3, 8])
-def test_step_host_matches_append_then_attend(env, groups):
+@pytest.mark.parametrize("groups, zero_copy", [(0, 1), (0, 0), (3, 1), (8, 1)])
+def test_step_host_matches_append_then_attend(env, groups, zero_copy):
     # groups > 0 forces the step to be cut into that many row groups whose copies and kernels overlap (what large
-    # steps do by themselves); pages, cache bits and outputs must not depend on the cut
+    # steps do by themselves); pages, cache bits and outputs must not depend on the cut.  A small step in one group
+    # is by default not copied at all (the kernels address the pinned host buffers); zero_copy = 0 takes the copies.
     tide, torch = env
     w = inputs.make_workload(1)
     kv_bits = [w.task_kv(b) for b in range(w.B)]
@@ -248,6 +249,7 @@ def test_step_host_matches_append_then_attend(env, groups):
     kv = tide.TideKV(w.Hq, w.Hkv, w.D, w.S, w.num_pages, w.max_tasks, w.max_pages_per_task, w.B, total_q,
                      free_order=w.free_order)
     kv.tune(tide.TUNE_HOST_STEP_CHUNKS, groups)
+    kv.tune(tide.TUNE_HOST_ZERO_COPY, zero_copy)
     for b in range(w.B):
         kv.alloc(int(w.task[b]))
     for b in range(w.B):
