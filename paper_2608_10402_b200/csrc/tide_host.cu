@@ -1497,12 +1497,20 @@ int tide_step_host(tide_kv_t* kv, int32_t layer, int32_t n_rows, const tide_row_
     if (cudaEventRecord(ev_start, st) != cudaSuccess || cudaStreamWaitEvent(s_in, ev_start, 0) != cudaSuccess) return TIDE_ERR_CUDA;
     if (cudaStreamWaitEvent(s_out, ev_start, 0) != cudaSuccess) return TIDE_ERR_CUDA;
   }
-  // rows [cut[c], cut[c+1]): up to the c+1-th share of the tokens, at least one row each
+  // rows [cut[c], cut[c+1]): up to the c+1-th share of the tokens, at least one row each.  The shares are equal but for
+  // the last two groups, which are a half and a fifth of a share: what follows the last copy in - that group's kernels
+  // and its copy out - is the part of the step that nothing overlaps, so it is kept short.
   int cut[kMaxHostChunks + 1];
   cut[0] = 0;
+  double share[kMaxHostChunks], share_sum = 0.0, share_acc = 0.0;
+  for (int c = 0; c < n_chunks; ++c) {
+    share[c] = (n_chunks >= 4 && c == n_chunks - 1) ? 0.2 : (n_chunks >= 4 && c == n_chunks - 2) ? 0.5 : 1.0;
+    share_sum += share[c];
+  }
   for (int c = 0; c < n_chunks; ++c) {
     int r1 = cut[c] + 1;
-    const long long goal = (long long)T * (c + 1) / n_chunks;
+    share_acc += share[c];
+    const long long goal = (long long)((double)T * share_acc / share_sum);
     while (r1 < n_rows && indptr[(size_t)r1 + 1] <= goal && n_rows - r1 > n_chunks - 1 - c) ++r1;
     cut[c + 1] = c == n_chunks - 1 ? n_rows : r1;
   }
